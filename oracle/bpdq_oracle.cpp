@@ -1,0 +1,187 @@
+// BPDQ reference checker ("oracle") -- TEST INFRASTRUCTURE ONLY.
+//
+// A plain, slow, single-threaded restatement of what the BPDQ weight-only linear layer
+// computes, written from the paper's definition of the variable grid.  It exists so that
+// the CUDA library can be checked element by element; it is never part of the product
+// path.  Only the test-suite, the smoke check and the benchmark's CPU-baseline leg may
+// load it.  It shares no source, header, table or helper with the CUDA library.
+//
+// What it follows:
+//   * Variable grid (Methodology, Eq. 1):  W^[r,j] = C0[r,G] + sum_{i=1..K} Ci[r,G] * Bi[r,j],
+//     Bi in {0,1}, G = floor(j / g)  (REP repeats a group coefficient over its g columns).
+//   * Candidate values of a group (Eq. 7; Appendix A.2: {0, c1, c2, c1+c2} for K = 2).
+//   * Quantized linear map (Section 3.1): the layer output is W^ applied to the activations,
+//     per token  y[m,r] = sum_j x[m,j] * W^[r,j].
+//
+// Readings where the paper is silent (it never states inference arithmetic):
+//   * coefficients are IEEE binary16 (forced by the bits-per-weight column of Table 1:
+//     K + 16 (K+1) / g);
+//   * decode: start from float(c0); for i = 1..K in that order, if the bit is set add
+//     float(ci) in IEEE binary32 (round to nearest even, no FMA, no reassociation); a clear
+//     bit adds nothing (so c0 = -0.0 with all bits clear stays -0.0); round once to
+//     binary16 (nearest even, overflow to infinity, subnormals kept);
+//   * linear: products and the running sum in binary64, sequential over j.  Alongside y the
+//     checker returns a[m,r] = sum_j |x[m,j] * W^[r,j]|, the scale of the accepted error.
+//
+// Pins (tests/test_oracle_*.py): hand-worked groups from Appendix A.2, the 2^K cardinality
+// bound, Proposition 1 (uniform grid as a special case, checked through an all-integer
+// route), all-zero / all-one plane closed forms, rounding ties and overflow, brute force on
+// tiny shapes against a differently structured decode, numpy's binary16 conversions, and a
+// float64 matrix product.  The acceptance bound on y (4e-3 * a + 1e-3) is stated by the
+// task, not by the paper: beyond that bound the y tolerance is "parity unpinned".
+//
+// oracle_unpack is an independent reader of the device blob layout, written from the
+// layout's description (not from the library's packer):
+//   planes : for block b = floor(j/128), plane i (0-based), row r: 16 bytes at byte offset
+//            ((b*K + i)*out + r)*16;  byte p of that unit holds the 8 columns
+//            128*b + 8*((p + r) mod 16) + t, t = bit number (LSB = 0);
+//   coefs  : after all planes; fp16 at byte offset ((G*(K+1) + i)*out + r)*2, i = 0 is c0.
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+
+namespace {
+
+float half_bits_to_float(uint16_t h) {
+    const uint32_t sign = (uint32_t)(h >> 15) & 1u;
+    const uint32_t expo = (uint32_t)(h >> 10) & 0x1Fu;
+    const uint32_t mant = (uint32_t)h & 0x3FFu;
+    double v;
+    if (expo == 0) {
+        v = std::ldexp((double)mant, -24);               // zero and subnormals: mant * 2^-24
+    } else if (expo == 31) {
+        v = mant ? std::nan("") : INFINITY;
+    } else {
+        v = std::ldexp((double)(mant + 1024u), (int)expo - 25);  // (1 + mant/1024) * 2^(expo-15)
+    }
+    float f = (float)v;                                   // every binary16 is exact in binary32
+    return sign ? -f : f;
+}
+
+// binary32 -> binary16, round to nearest even.
+uint16_t float_to_half_bits(float f) {
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    const uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+    const uint32_t absu = u & 0x7FFFFFFFu;
+    if (absu > 0x7F800000u) return (uint16_t)(sign | 0x7E00u);            // NaN
+    if (absu == 0x7F800000u) return (uint16_t)(sign | 0x7C00u);           // infinity
+    // Work on the magnitude as an exact rational: value = m * 2^e with integer m.
+    const int e32 = (int)(absu >> 23);
+    uint64_t m = absu & 0x7FFFFFu;
+    int e;                        // value = m * 2^e
+    if (e32 == 0) { e = -149; } else { m |= 0x800000u; e = e32 - 150; }
+    if (m == 0) return sign;
+    // Target: value = q * 2^-24 for subnormal halves (q < 1024), or q * 2^(E-25) with
+    // 1024 <= q < 2048 for normal halves with biased exponent E in 1..30.
+    // Find the unbiased position of the leading bit.
+    int lead = 63;
+    while (!((m >> lead) & 1)) --lead;
+    int top = lead + e;           // value in [2^top, 2^(top+1))
+    int ulp_exp = (top < -14) ? -24 : top - 10;   // exponent of one half-precision ulp here
+    // q = round_to_nearest_even(m * 2^(e - ulp_exp))
+    int shift = ulp_exp - e;      // >= 0 means we drop `shift` low bits of m
+    uint64_t q;
+    if (shift <= 0) {
+        q = m << (-shift);
+    } else if (shift > 63) {
+        q = 0;
+    } else {
+        const uint64_t keep = m >> shift;
+        const uint64_t rem = m & ((1ull << shift) - 1);
+        const uint64_t half = 1ull << (shift - 1);
+        q = keep;
+        if (rem > half || (rem == half && (keep & 1))) q += 1;
+    }
+    if (top < -14) {
+        // subnormal range; q may round up to 1024, which is exactly the smallest normal.
+        return (uint16_t)(sign | (uint16_t)q);
+    }
+    int E = top + 15;
+    if (q == 2048) { q = 1024; E += 1; }
+    if (E >= 31) return (uint16_t)(sign | 0x7C00u);                        // overflow
+    return (uint16_t)(sign | (uint16_t)(E << 10) | (uint16_t)(q - 1024));
+}
+
+inline uint16_t decode_one(const uint8_t* bits, const uint16_t* coef, int64_t out, int64_t in,
+                           int K, int64_t ngroups, int64_t r, int64_t j, int64_t G) {
+    // Eq. 1 for one weight.  `volatile` keeps every binary32 addition a separate, rounded step.
+    volatile float acc = half_bits_to_float(coef[(0 * out + r) * ngroups + G]);
+    for (int i = 1; i <= K; ++i) {
+        if (bits[((int64_t)(i - 1) * out + r) * in + j]) {
+            const float ci = half_bits_to_float(coef[((int64_t)i * out + r) * ngroups + G]);
+            acc = acc + ci;
+        }
+    }
+    return float_to_half_bits(acc);
+}
+
+}  // namespace
+
+extern "C" {
+
+// Conversions, exported so the tests can pin them against an independent implementation.
+float oracle_half_to_float(uint16_t h) { return half_bits_to_float(h); }
+uint16_t oracle_float_to_half(float f) { return float_to_half_bits(f); }
+
+// bits [K][out][in] (0/1), coef [K+1][out][in/g] fp16 bits -> w [out][in] fp16 bits.
+int oracle_dequant(const uint8_t* bits, const uint16_t* coef, int64_t out, int64_t in, int K,
+                   int64_t g, uint16_t* w) {
+    if (!bits || !coef || !w || out <= 0 || in <= 0 || K < 1 || g <= 0 || in % g) return 1;
+    const int64_t ngroups = in / g;
+    for (int64_t r = 0; r < out; ++r)
+        for (int64_t j = 0; j < in; ++j)
+            w[r * in + j] = decode_one(bits, coef, out, in, K, ngroups, r, j, j / g);
+    return 0;
+}
+
+// x [M][in] fp16 bits -> y [M][out], a [M][out] in binary64 (a may be NULL).
+int oracle_linear(const uint8_t* bits, const uint16_t* coef, const uint16_t* x, int64_t out,
+                  int64_t in, int K, int64_t g, int64_t M, double* y, double* a) {
+    if (!bits || !coef || !x || !y || out <= 0 || in <= 0 || K < 1 || g <= 0 || in % g || M < 0)
+        return 1;
+    const int64_t ngroups = in / g;
+    for (int64_t r = 0; r < out; ++r) {
+        for (int64_t m = 0; m < M; ++m) { y[m * out + r] = 0.0; if (a) a[m * out + r] = 0.0; }
+        for (int64_t j = 0; j < in; ++j) {
+            const double wj = (double)half_bits_to_float(
+                decode_one(bits, coef, out, in, K, ngroups, r, j, j / g));
+            for (int64_t m = 0; m < M; ++m) {
+                const double p = (double)half_bits_to_float(x[m * in + j]) * wj;
+                y[m * out + r] += p;
+                if (a) a[m * out + r] += std::fabs(p);
+            }
+        }
+    }
+    return 0;
+}
+
+// Device blob -> logical tensors (layout described in the header comment of this file).
+int oracle_unpack(const uint8_t* blob, int64_t out, int64_t in, int K, int64_t g, uint8_t* bits,
+                  uint16_t* coef) {
+    if (!blob || !bits || !coef || out <= 0 || in <= 0 || K < 1 || g <= 0 || in % g || in % 128)
+        return 1;
+    const int64_t nblocks = in / 128, ngroups = in / g;
+    for (int64_t b = 0; b < nblocks; ++b)
+        for (int i = 0; i < K; ++i)
+            for (int64_t r = 0; r < out; ++r) {
+                const uint8_t* unit = blob + ((b * K + i) * out + r) * 16;
+                for (int p = 0; p < 16; ++p) {
+                    const int64_t chunk = (p + r) % 16;
+                    for (int t = 0; t < 8; ++t)
+                        bits[((int64_t)i * out + r) * in + 128 * b + 8 * chunk + t] =
+                            (uint8_t)((unit[p] >> t) & 1);
+                }
+            }
+    const uint8_t* cbase = blob + out * in * K / 8;
+    for (int64_t G = 0; G < ngroups; ++G)
+        for (int i = 0; i <= K; ++i)
+            for (int64_t r = 0; r < out; ++r) {
+                uint16_t v;
+                std::memcpy(&v, cbase + ((G * (K + 1) + i) * out + r) * 2, 2);
+                coef[((int64_t)i * out + r) * ngroups + G] = v;
+            }
+    return 0;
+}
+
+}  // extern "C"

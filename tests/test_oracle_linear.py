@@ -1,0 +1,81 @@
+"""Pins of the reference checker's linear map y = x * W^T and of its blob reader.  CPU only."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2602_04163_b200 import synth
+
+
+def f16(bits):
+    return np.asarray(bits, dtype=np.uint16).view(np.float16)
+
+
+@pytest.mark.parametrize("K,g,out,in_,M", [(2, 128, 48, 384, 1), (3, 128, 40, 256, 3), (2, 64, 24, 192, 2),
+                                            (4, 256, 8, 512, 1)])
+def test_linear_matches_float64_matmul(K, g, out, in_, M):
+    """Special case that reduces to a library routine: dequantize, then a float64 matrix product.
+    Non-square shapes with M != out catch a transposed operand or a swapped output index."""
+    bits = synth.plane_bits(21, out, in_, K)
+    coef = synth.coefficients(21, out, in_, K, g)
+    x = synth.activations(22, M, in_)
+    w = f16(oracle.dequant(bits, coef, g)).astype(np.float64)
+    xf = f16(x).astype(np.float64)
+    y, a = oracle.linear(bits, coef, x, g)
+    assert y.shape == (M, out)
+    assert np.allclose(y, xf @ w.T, rtol=1e-12, atol=1e-12)
+    assert np.allclose(a, np.abs(xf) @ np.abs(w).T, rtol=1e-12, atol=1e-12)
+    assert np.all(a >= np.abs(y) - 1e-12)
+
+
+def test_linear_one_hot_activation_reads_one_column():
+    """x = e_j picks column j of W^: y[0, r] = W^[r, j] exactly."""
+    K, g, out, in_ = 2, 128, 16, 256
+    bits = synth.plane_bits(1, out, in_, K)
+    coef = synth.coefficients(1, out, in_, K, g)
+    w = f16(oracle.dequant(bits, coef, g)).astype(np.float64)
+    for j in (0, 1, 127, 128, 255):
+        x = np.zeros((1, in_), dtype=np.float16)
+        x[0, j] = 1.0
+        y, a = oracle.linear(bits, coef, x.view(np.uint16), g)
+        assert np.array_equal(y[0], w[:, j])
+        assert np.array_equal(a[0], np.abs(w[:, j]))
+
+
+def test_linear_add_only_identity():
+    """y_r = sum_G [ c0*X_G + sum_i ci * S_i ],  S_i = sum of x over the set bits of plane i
+    (the add-only form the paper names for custom hardware) agrees with the definition up to the
+    one binary16 rounding of each weight."""
+    K, g, out, in_ = 3, 128, 32, 512
+    bits = synth.plane_bits(9, out, in_, K)
+    coef = synth.coefficients(9, out, in_, K, g)
+    x = synth.activations(9, 1, in_)
+    y, a = oracle.linear(bits, coef, x, g)
+    xf = f16(x).astype(np.float64)[0]
+    cf = f16(coef).astype(np.float64)
+    alt = np.zeros(out)
+    for G in range(in_ // g):
+        xs = xf[G * g:(G + 1) * g]
+        alt += cf[0, :, G] * xs.sum()
+        for i in range(K):
+            alt += cf[i + 1, :, G] * (bits[i, :, G * g:(G + 1) * g] * xs).sum(axis=1)
+    assert np.all(np.abs(alt - y[0]) <= 2.0 ** -11 * a[0] + 1e-12)
+
+
+def test_unpack_reads_documented_layout():
+    """Build a blob by hand from the layout description and read it back."""
+    K, g, out, in_ = 2, 128, 32, 256
+    bits = synth.plane_bits(4, out, in_, K)
+    coef = synth.coefficients(4, out, in_, K, g)
+    nblk = in_ // 128
+    planes = np.zeros((nblk, K, out, 16), dtype=np.uint8)
+    for b in range(nblk):
+        for i in range(K):
+            for r in range(out):
+                for p in range(16):
+                    c = (p + r) % 16
+                    cols = bits[i, r, 128 * b + 8 * c: 128 * b + 8 * c + 8]
+                    planes[b, i, r, p] = sum(int(v) << t for t, v in enumerate(cols))
+    cblob = np.transpose(coef, (2, 0, 1)).copy()          # [G][i][r]
+    blob = np.concatenate([planes.reshape(-1), cblob.reshape(-1).view(np.uint8)])
+    b2, c2 = oracle.unpack(blob, out, in_, K, g)
+    assert np.array_equal(b2, bits) and np.array_equal(c2, coef)
