@@ -1,0 +1,156 @@
+/* bpdq.h -- C ABI of the BPDQ weight-only linear layer for NVIDIA B200 (sm_100a).
+ *
+ * The operation (paper: Methodology, Eq. 1; candidate values Eq. 7; Appendix A.2):
+ *
+ *     W^[r, j] = C0[r, G] + sum_{i=1..K} Ci[r, G] * Bi[r, j],   Bi in {0,1},  G = floor(j / g)
+ *
+ * a "variable grid": K bit-planes Bi of shape [out][in] plus K+1 scalar coefficients per
+ * (output row r, input group G of g columns).  The layer output is the quantized weight
+ * applied to the activations (paper: Section 3.1, the output-aligned objective compares W X
+ * with W^ X), per token
+ *
+ *     y[m, r] = sum_j x[m, j] * W^[r, j].
+ *
+ * The paper fixes no inference arithmetic.  This library uses: coefficients stored as IEEE
+ * binary16 (the paper's bits-per-weight figures, K + 16 (K+1) / g, leave room for nothing
+ * else); a weight is decoded as float(c0), then for i = 1..K in order "if the bit is set add
+ * float(ci)" in binary32, then rounded once to binary16 (bpdq_dequant returns exactly that
+ * bit pattern); x and y are binary16, accumulation is binary32.
+ *
+ * Conventions
+ *   - every function returns a status code (below) and never throws or aborts;
+ *     bpdq_last_error() gives a thread-local text for the last non-OK status;
+ *   - "host" / "device" says where a pointer must live.  Device pointers must be 16-byte
+ *     aligned, tensors are dense row-major;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *     that take a stream only enqueue work and do not synchronise, unless stated;
+ *   - a handle owns its device copy of the packed weights and a scratch workspace.  Two calls
+ *     on the same handle must not overlap on the GPU (issue them on one stream);
+ *   - supported shapes: K in {1,2,3,4}; g in {64,128,256}; in % 128 == 0 and in % g == 0;
+ *     out % 16 == 0.  Anything else is BPDQ_ERR_UNSUPPORTED.
+ *
+ * Logical tensors (what pack/unpack exchange with the caller)
+ *   bits : uint8  [K][out][in], values 0/1; bits[i] is the paper's plane B_{i+1}
+ *   coef : uint16 [K+1][out][in/g], binary16 bit patterns; coef[0] is C0, coef[i] is Ci
+ *
+ * Packed blob (what lives in device memory), bpdq_packed_bytes() bytes, no padding:
+ *   planes, then coefficients.
+ *   planes : 32-bit words run along the input dimension; four words (128 columns, a "block")
+ *            of one plane and one row form a 16-byte unit, and for a fixed block and plane
+ *            the units of consecutive rows are adjacent, so that a warp reads 32 rows with one
+ *            coalesced 512-byte request and a 128-row tile is one contiguous 2 KB run:
+ *              unit(b, i, r) at byte ((b*K + i)*out + r)*16,   b = floor(j/128), i 0-based.
+ *            Inside a unit the sixteen 8-column bytes are rotated by the row number: byte p
+ *            holds columns 128*b + 8*((p + r) mod 16) + t, bit t (LSB = 0).  Rows that a
+ *            half-warp handles together therefore index sixteen different 8-column look-up
+ *            tables at every step.
+ *   coefs  : binary16 at byte planes_bytes + ((G*(K+1) + i)*out + r)*2.
+ */
+#ifndef BPDQ_H_
+#define BPDQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define BPDQ_API __attribute__((visibility("default")))
+#else
+#define BPDQ_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct bpdq_handle_s* bpdq_handle_t;
+
+enum {
+    BPDQ_OK = 0,
+    BPDQ_ERR_INVALID = 1,     /* null / misaligned pointer, bad size, M out of range          */
+    BPDQ_ERR_UNSUPPORTED = 2, /* shape outside the supported set, or no sm_100 device         */
+    BPDQ_ERR_ALLOC = 3,       /* device or host allocation failed                             */
+    BPDQ_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed                          */
+    BPDQ_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (read by bpdq_get_status) */
+};
+
+/* Which kernel bpdq_linear_ex runs. */
+enum {
+    BPDQ_KERNEL_AUTO = 0,     /* dispatch on M (what bpdq_linear does)                        */
+    BPDQ_KERNEL_GEMV = 1,     /* look-up-table kernel, M <= BPDQ_GEMV_MAX_M                   */
+    BPDQ_KERNEL_GEMM = 2,     /* tensor-core kernel (TMA + tcgen05), any M >= 1               */
+    BPDQ_KERNEL_GEMV_SIMPLE = 3 /* one-bit-at-a-time kernel kept as an on-device cross-check  */
+};
+
+#define BPDQ_GEMV_MAX_M 16
+
+/* Storage accounting (paper: Table 1, column BPW = K + 16 (K+1) / g bits per weight).
+ * Bytes of the packed blob: out*in*K/8 + out*(in/g)*(K+1)*2.  Returns 0 for an unsupported
+ * shape.  Host only, no CUDA call. */
+BPDQ_API size_t bpdq_packed_bytes(int out, int in, int K, int group);
+
+/* Host packer: logical tensors -> blob (layout above).  All pointers are host memory;
+ * `blob` is caller-owned with bpdq_packed_bytes() bytes.  Every bit value must be 0 or 1
+ * (BPDQ_ERR_INVALID otherwise).  Defines the storage of Eq. 1's B_i and C_i. */
+BPDQ_API int bpdq_pack(const uint8_t* bits, const uint16_t* coef, int out, int in, int K, int group,
+              void* blob);
+
+/* Inverse of bpdq_pack: blob -> logical tensors.  unpack(pack(b, c)) == (b, c). */
+BPDQ_API int bpdq_unpack(const void* blob, int out, int in, int K, int group, uint8_t* bits,
+                uint16_t* coef);
+
+/* Creates a layer on the current CUDA device.  `host_blob` (host memory, bpdq_packed_bytes()
+ * bytes) is copied to the device; if it is NULL the blob is generated on the device from
+ * `seed` with the counter-based generator of the synthetic workloads (plane bits iid
+ * Bernoulli(1/2); c0 ~ N(0, 0.02); c1, c2 ~ U(0.005, 0.05); c3.. ~ U(0.002, 0.02)), which
+ * reproduces the host generator bit for bit.  `max_M` (>= 1) bounds the token count of later
+ * bpdq_linear calls and sizes the workspace.  Synchronises the device.  On failure *h is
+ * NULL. */
+BPDQ_API int bpdq_create(bpdq_handle_t* h, int out, int in, int K, int group, const void* host_blob,
+                uint64_t seed, int max_M);
+
+/* Eq. 1 materialised: writes W^ as binary16 [out][in] row-major to `w_fp16_dev` (device,
+ * caller-owned, out*in*2 bytes).  Bit-exact with the decode rule stated at the top. */
+BPDQ_API int bpdq_dequant(bpdq_handle_t h, void* w_fp16_dev, void* stream);
+
+/* The quantized linear map y = x * W^T (paper: Eq. 1 applied to activations, Section 3.1).
+ * x: device binary16 [M][in]; y: device binary16 [M][out]; 0 <= M <= max_M.  M == 0 returns
+ * BPDQ_OK without a launch.  Picks the look-up-table kernel for small M and the tensor-core
+ * kernel above the handle's dispatch threshold.  x and y must not alias. */
+BPDQ_API int bpdq_linear(bpdq_handle_t h, const void* x_fp16_dev, void* y_fp16_dev, int M, void* stream);
+
+/* Same map with the kernel chosen by the caller (BPDQ_KERNEL_*).  BPDQ_KERNEL_GEMV with
+ * M > BPDQ_GEMV_MAX_M is BPDQ_ERR_INVALID. */
+BPDQ_API int bpdq_linear_ex(bpdq_handle_t h, const void* x_fp16_dev, void* y_fp16_dev, int M, int kernel,
+                   void* stream);
+
+/* Same map for callers whose activations live in HOST memory: copies x (host, [M][in]) to a
+ * handle-owned staging buffer, runs bpdq_linear, copies y back to `y_fp16_host` and waits for
+ * the stream.  Pinned host memory makes the copies asynchronous up to that wait. */
+BPDQ_API int bpdq_linear_host(bpdq_handle_t h, const void* x_fp16_host, void* y_fp16_host, int M,
+                     void* stream);
+
+/* Sets the largest M that bpdq_linear sends to the look-up-table kernel (0 = always use the
+ * tensor-core kernel; at most BPDQ_GEMV_MAX_M). */
+BPDQ_API int bpdq_set_gemv_max_m(bpdq_handle_t h, int max_gemv_m);
+
+/* Copies the device blob back to host memory (bpdq_packed_bytes() bytes); synchronises. */
+BPDQ_API int bpdq_read_blob(bpdq_handle_t h, void* host_blob);
+
+/* Waits for `stream` and returns the handle's device status word: BPDQ_OK, or
+ * BPDQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up (the result of that call is
+ * then undefined; the context stays usable).  Clears the word. */
+BPDQ_API int bpdq_get_status(bpdq_handle_t h, void* stream);
+
+/* Number of kernels this handle has launched since creation (bookkeeping for benchmarks). */
+BPDQ_API int bpdq_launch_count(bpdq_handle_t h, uint64_t* count);
+
+/* Frees everything the handle owns; synchronises the device.  NULL is BPDQ_OK. */
+BPDQ_API int bpdq_destroy(bpdq_handle_t h);
+
+/* Text of the calling thread's last non-OK status ("" if none). */
+BPDQ_API const char* bpdq_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BPDQ_H_ */

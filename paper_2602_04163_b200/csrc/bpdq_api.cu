@@ -1,0 +1,193 @@
+// C ABI entry points that own device state: create / destroy / dequant / linear and friends.
+// Argument checks happen here; kernels live in their own translation units.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "bpdq_internal.h"
+
+using namespace bpdq;
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int cuda_fail(const char* what, cudaError_t e) {
+    return set_error(BPDQ_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+void free_handle(bpdq_handle_s* h) {
+    if (!h) return;
+    if (h->d_blob) cudaFree(h->d_blob);
+    if (h->d_ws) cudaFree(h->d_ws);
+    if (h->d_counters) cudaFree(h->d_counters);
+    if (h->d_status) cudaFree(h->d_status);
+    if (h->d_xstage) cudaFree(h->d_xstage);
+    if (h->d_ystage) cudaFree(h->d_ystage);
+    delete h;
+}
+
+int check_linear_args(bpdq_handle_s* h, const void* x, void* y, int M, const char* who) {
+    if (!h) return set_error(BPDQ_ERR_INVALID, "%s: null handle", who);
+    if (M < 0 || M > h->max_M) return set_error(BPDQ_ERR_INVALID, "%s: M=%d outside [0, max_M=%d]", who, M, h->max_M);
+    if (M == 0) return BPDQ_OK;
+    if (!x || !y) return set_error(BPDQ_ERR_INVALID, "%s: null pointer", who);
+    return BPDQ_OK;
+}
+
+}  // namespace
+
+extern "C" int bpdq_create(bpdq_handle_t* hp, int out, int in, int K, int group, const void* host_blob,
+                           uint64_t seed, int max_M) {
+    if (!hp) return set_error(BPDQ_ERR_INVALID, "bpdq_create: null handle pointer");
+    *hp = nullptr;
+    if (max_M < 1) return set_error(BPDQ_ERR_INVALID, "bpdq_create: max_M=%d must be >= 1", max_M);
+    if (!shape_supported(out, in, K, group))
+        return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_create: unsupported shape out=%d in=%d K=%d g=%d", out, in, K, group);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_create: no CUDA device (%s)", cudaGetErrorString(e));
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, dev);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDeviceProperties", e);
+    if (prop.major != 10)
+        return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_create: device is sm_%d%d, this library is built for sm_100a only",
+                         prop.major, prop.minor);
+
+    bpdq_handle_s* h = new (std::nothrow) bpdq_handle_s();
+    if (!h) return set_error(BPDQ_ERR_ALLOC, "bpdq_create: host allocation failed");
+    std::memset(h, 0, sizeof(*h));
+    h->out = out; h->in = in; h->K = K; h->group = group; h->max_M = max_M; h->device = dev;
+    h->sm_count = prop.multiProcessorCount;
+    h->planes_bytes = planes_bytes(out, in, K);
+    h->blob_bytes = h->planes_bytes + coefs_bytes(out, in, K, group);
+    h->ws_bytes = gemv_workspace_bytes(out, in, K, group, max_M, h->sm_count);
+    h->n_counters = gemv_counter_count(out);
+    h->gemv_max_m = 2;
+
+    const size_t stage_x = (size_t)max_M * in * 2, stage_y = (size_t)max_M * out * 2;
+    if ((e = cudaMalloc(&h->d_blob, h->blob_bytes)) != cudaSuccess ||
+        (e = cudaMalloc(&h->d_ws, h->ws_bytes ? h->ws_bytes : 16)) != cudaSuccess ||
+        (e = cudaMalloc(&h->d_counters, (h->n_counters ? h->n_counters : 1) * sizeof(unsigned))) != cudaSuccess ||
+        (e = cudaMalloc(&h->d_status, sizeof(int))) != cudaSuccess ||
+        (e = cudaMalloc(&h->d_xstage, stage_x)) != cudaSuccess ||
+        (e = cudaMalloc(&h->d_ystage, stage_y)) != cudaSuccess) {
+        free_handle(h);
+        cudaGetLastError();
+        return set_error(BPDQ_ERR_ALLOC, "bpdq_create: cudaMalloc failed (%s)", cudaGetErrorString(e));
+    }
+    cudaMemset(h->d_counters, 0, (h->n_counters ? h->n_counters : 1) * sizeof(unsigned));
+    cudaMemset(h->d_status, 0, sizeof(int));
+    int rc = BPDQ_OK;
+    if (host_blob) {
+        e = cudaMemcpy(h->d_blob, host_blob, h->blob_bytes, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) rc = cuda_fail("bpdq_create: blob copy", e);
+    } else {
+        rc = launch_fill(h, seed, nullptr);
+    }
+    if (rc == BPDQ_OK) {
+        e = cudaDeviceSynchronize();
+        if (e != cudaSuccess) rc = cuda_fail("bpdq_create: synchronize", e);
+    }
+    if (rc != BPDQ_OK) { free_handle(h); return rc; }
+    *hp = h;
+    return BPDQ_OK;
+}
+
+extern "C" int bpdq_destroy(bpdq_handle_t h) {
+    if (!h) return BPDQ_OK;
+    cudaError_t e = cudaDeviceSynchronize();
+    free_handle(h);
+    if (e != cudaSuccess) return cuda_fail("bpdq_destroy: synchronize", e);
+    return BPDQ_OK;
+}
+
+extern "C" int bpdq_dequant(bpdq_handle_t h, void* w, void* stream) {
+    if (!h) return set_error(BPDQ_ERR_INVALID, "bpdq_dequant: null handle");
+    if (!w) return set_error(BPDQ_ERR_INVALID, "bpdq_dequant: null output pointer");
+    if (!aligned16(w)) return set_error(BPDQ_ERR_INVALID, "bpdq_dequant: output pointer not 16-byte aligned");
+    return launch_dequant(h, w, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int bpdq_linear_ex(bpdq_handle_t h, const void* x, void* y, int M, int kernel, void* stream) {
+    int rc = check_linear_args(h, x, y, M, "bpdq_linear");
+    if (rc != BPDQ_OK || M == 0) return rc;
+    if (!aligned16(x) || !aligned16(y))
+        return set_error(BPDQ_ERR_INVALID, "bpdq_linear: x and y must be 16-byte aligned");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (kernel == BPDQ_KERNEL_AUTO) {
+        const bool gv = gemv_supported(h->out, h->in, h->K, h->group);
+        const bool gm = gemm_supported(h->out, h->in, h->K, h->group);
+        if (gv && (M <= h->gemv_max_m || !gm) && M <= BPDQ_GEMV_MAX_M) kernel = BPDQ_KERNEL_GEMV;
+        else if (gm) kernel = BPDQ_KERNEL_GEMM;
+        else kernel = BPDQ_KERNEL_GEMV_SIMPLE;
+    }
+    switch (kernel) {
+        case BPDQ_KERNEL_GEMV:
+            if (M > BPDQ_GEMV_MAX_M)
+                return set_error(BPDQ_ERR_INVALID, "bpdq_linear: look-up-table kernel takes M <= %d, got %d", BPDQ_GEMV_MAX_M, M);
+            if (!gemv_supported(h->out, h->in, h->K, h->group))
+                return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear: look-up-table kernel does not cover K=%d g=%d", h->K, h->group);
+            return launch_gemv(h, x, y, M, s);
+        case BPDQ_KERNEL_GEMM:
+            if (!gemm_supported(h->out, h->in, h->K, h->group))
+                return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear: tensor-core kernel does not cover K=%d g=%d", h->K, h->group);
+            return launch_gemm(h, x, y, M, s);
+        case BPDQ_KERNEL_GEMV_SIMPLE:
+            return launch_gemv_simple(h, x, y, M, s);
+        default:
+            return set_error(BPDQ_ERR_INVALID, "bpdq_linear: unknown kernel id %d", kernel);
+    }
+}
+
+extern "C" int bpdq_linear(bpdq_handle_t h, const void* x, void* y, int M, void* stream) {
+    return bpdq_linear_ex(h, x, y, M, BPDQ_KERNEL_AUTO, stream);
+}
+
+extern "C" int bpdq_linear_host(bpdq_handle_t h, const void* x_host, void* y_host, int M, void* stream) {
+    int rc = check_linear_args(h, x_host, y_host, M, "bpdq_linear_host");
+    if (rc != BPDQ_OK || M == 0) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(h->d_xstage, x_host, (size_t)M * h->in * 2, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail("bpdq_linear_host: copy in", e);
+    rc = bpdq_linear_ex(h, h->d_xstage, h->d_ystage, M, BPDQ_KERNEL_AUTO, stream);
+    if (rc != BPDQ_OK) return rc;
+    e = cudaMemcpyAsync(y_host, h->d_ystage, (size_t)M * h->out * 2, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail("bpdq_linear_host: copy out", e);
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail("bpdq_linear_host: synchronize", e);
+    return BPDQ_OK;
+}
+
+extern "C" int bpdq_set_gemv_max_m(bpdq_handle_t h, int max_gemv_m) {
+    if (!h) return set_error(BPDQ_ERR_INVALID, "bpdq_set_gemv_max_m: null handle");
+    if (max_gemv_m < 0 || max_gemv_m > BPDQ_GEMV_MAX_M)
+        return set_error(BPDQ_ERR_INVALID, "bpdq_set_gemv_max_m: %d outside [0, %d]", max_gemv_m, BPDQ_GEMV_MAX_M);
+    h->gemv_max_m = max_gemv_m;
+    return BPDQ_OK;
+}
+
+extern "C" int bpdq_read_blob(bpdq_handle_t h, void* host_blob) {
+    if (!h || !host_blob) return set_error(BPDQ_ERR_INVALID, "bpdq_read_blob: null pointer");
+    cudaError_t e = cudaMemcpy(host_blob, h->d_blob, h->blob_bytes, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail("bpdq_read_blob", e);
+    return BPDQ_OK;
+}
+
+extern "C" int bpdq_get_status(bpdq_handle_t h, void* stream) {
+    if (!h) return set_error(BPDQ_ERR_INVALID, "bpdq_get_status: null handle");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int st = 0;
+    cudaError_t e = cudaMemcpyAsync(&st, h->d_status, sizeof(int), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->d_status, 0, sizeof(int), s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail("bpdq_get_status", e);
+    if (st != BPDQ_OK) return set_error(st, "a device-side bounded wait expired (status %d)", st);
+    return BPDQ_OK;
+}
+
+extern "C" int bpdq_launch_count(bpdq_handle_t h, uint64_t* count) {
+    if (!h || !count) return set_error(BPDQ_ERR_INVALID, "bpdq_launch_count: null pointer");
+    *count = h->launches;
+    return BPDQ_OK;
+}

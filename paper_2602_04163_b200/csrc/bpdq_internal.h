@@ -1,0 +1,65 @@
+// Internal declarations shared by the translation units of libbpdq (not part of the ABI).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "bpdq.h"
+
+#if defined(__CUDACC__)
+#define BPDQ_HD __host__ __device__ __forceinline__
+#else
+#define BPDQ_HD inline
+#endif
+
+namespace bpdq {
+
+constexpr int kBlockCols = 128;   // columns covered by one 16-byte plane unit
+constexpr int kUnitBytes = 16;
+
+// Byte offset of the 16-byte unit of (block b, plane i (0-based), row r).
+BPDQ_HD size_t plane_unit_offset(int64_t b, int i, int64_t r, int K, int64_t out) {
+    return (size_t)(((b * K + i) * out + r) * kUnitBytes);
+}
+// Byte offset (inside the coefficient section) of coefficient i of (group G, row r).
+BPDQ_HD size_t coef_offset(int64_t G, int i, int64_t r, int K, int64_t out) {
+    return (size_t)(((G * (K + 1) + i) * out + r) * 2);
+}
+BPDQ_HD size_t planes_bytes(int64_t out, int64_t in, int K) { return (size_t)(out * in * K / 8); }
+BPDQ_HD size_t coefs_bytes(int64_t out, int64_t in, int K, int64_t g) {
+    return (size_t)(out * (in / g) * (K + 1) * 2);
+}
+
+bool shape_supported(int out, int in, int K, int group);
+int set_error(int code, const char* fmt, ...);
+
+}  // namespace bpdq
+
+struct bpdq_handle_s {
+    int out, in, K, group, max_M, device;
+    int sm_count;
+    uint8_t* d_blob;          // planes then coefficients
+    size_t blob_bytes, planes_bytes;
+    float* d_ws;              // split-K partial sums
+    size_t ws_bytes;
+    unsigned* d_counters;     // one arrival counter per 32-row block (self-resetting)
+    size_t n_counters;
+    int* d_status;            // device status word
+    void* d_xstage;           // staging for bpdq_linear_host
+    void* d_ystage;
+    int gemv_max_m;
+    uint64_t launches;
+};
+
+// Kernel launchers (each returns a BPDQ_* status; all asynchronous on `stream`).
+namespace bpdq {
+int launch_fill(bpdq_handle_s* h, uint64_t seed, cudaStream_t stream);
+int launch_dequant(bpdq_handle_s* h, void* w, cudaStream_t stream);
+int launch_gemv_simple(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
+int launch_gemv(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
+int launch_gemm(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
+size_t gemv_workspace_bytes(int out, int in, int K, int group, int max_M, int sm_count);
+size_t gemv_counter_count(int out);
+bool gemv_supported(int out, int in, int K, int group);
+bool gemm_supported(int out, int in, int K, int group);
+}  // namespace bpdq

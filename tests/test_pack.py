@@ -1,0 +1,77 @@
+"""Host packer: round trip, agreement with the checker's independent blob reader, storage accounting."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2602_04163_b200 import binding, synth
+
+
+@pytest.mark.parametrize("K,g,out,in_", [(2, 128, 48, 384), (3, 128, 32, 256), (1, 64, 16, 128), (4, 256, 64, 512),
+                                          (2, 64, 80, 256)])
+def test_round_trip_and_independent_reader(K, g, out, in_):
+    bits = synth.plane_bits(3, out, in_, K)
+    coef = synth.coefficients(3, out, in_, K, g)
+    blob = binding.bpdq_pack(bits, coef, g)
+    assert blob.size == out * in_ * K // 8 + out * (in_ // g) * (K + 1) * 2
+    b2, c2 = binding.bpdq_unpack(blob, out, in_, K, g)
+    assert np.array_equal(b2, bits) and np.array_equal(c2, coef)
+    b3, c3 = oracle.unpack(blob, out, in_, K, g)          # written from the layout text, not from the packer
+    assert np.array_equal(b3, bits) and np.array_equal(c3, coef)
+
+
+def test_one_hot_bits_land_where_the_layout_says():
+    """One set bit at a time: catches any permutation error of plane, row, block, byte or bit."""
+    K, g, out, in_ = 2, 128, 32, 256
+    coef = np.zeros((K + 1, out, in_ // g), dtype=np.uint16)
+    rng = np.random.default_rng(0)
+    for _ in range(200):
+        i, r, j = int(rng.integers(K)), int(rng.integers(out)), int(rng.integers(in_))
+        bits = np.zeros((K, out, in_), dtype=np.uint8)
+        bits[i, r, j] = 1
+        blob = binding.bpdq_pack(bits, coef, g)
+        nz = np.flatnonzero(blob)
+        assert nz.size == 1
+        b, c, t = j // 128, (j % 128) // 8, j % 8
+        p = (c - r) % 16
+        assert nz[0] == ((b * K + i) * out + r) * 16 + p and blob[nz[0]] == 1 << t
+
+
+def test_coefficient_placement():
+    K, g, out, in_ = 3, 64, 16, 128
+    bits = np.zeros((K, out, in_), dtype=np.uint8)
+    coef = np.arange((K + 1) * out * (in_ // g), dtype=np.uint16).reshape(K + 1, out, in_ // g) + 1
+    blob = binding.bpdq_pack(bits, coef, g)
+    c = blob[out * in_ * K // 8:].view(np.uint16).reshape(in_ // g, K + 1, out)
+    assert np.array_equal(np.transpose(c, (1, 2, 0)), coef)
+
+
+def test_bits_per_weight_matches_table_1(golden_dir):
+    rows = [ln.split() for ln in open(f"{golden_dir}/bits_per_weight.txt") if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 6
+    for K, g, printed in rows:
+        K, g = int(K), int(g)
+        out, in_ = 256, 1024
+        bpw = 8 * binding.bpdq_packed_bytes(out, in_, K, g) / (out * in_)
+        assert bpw == K + 16 * (K + 1) / g                  # exact: no padding, no header
+        assert abs(bpw - float(printed)) <= 0.005 + 1e-12   # the table rounds to two decimals
+
+
+def test_workload_byte_counts():
+    """Useful bytes of the benchmark layers (planes + binary16 coefficients, g = 128)."""
+    assert binding.bpdq_packed_bytes(4096, 4096, 2, 128) == 4_980_736
+    assert sum(binding.bpdq_packed_bytes(o, i, 2, 128) for _, o, i in synth.QWEN25_7B_LAYER) == 69_185_536
+    assert sum(binding.bpdq_packed_bytes(o, i, 2, 128) for _, o, i in synth.QWEN25_72B_LAYER) == 260_554_752
+    assert sum(binding.bpdq_packed_bytes(o, i, 3, 128) for _, o, i in synth.QWEN25_72B_LAYER) == 383_975_424
+
+
+def test_rejects_bad_input():
+    assert binding.bpdq_packed_bytes(100, 256, 2, 128) == 0       # out % 16
+    assert binding.bpdq_packed_bytes(128, 200, 2, 128) == 0       # in % 128
+    assert binding.bpdq_packed_bytes(128, 256, 5, 128) == 0
+    assert binding.bpdq_packed_bytes(128, 256, 2, 32) == 0
+    assert binding.bpdq_packed_bytes(128, 384, 2, 256) == 0       # in % g
+    bits = np.zeros((2, 16, 128), dtype=np.uint8)
+    bits[1, 3, 5] = 2
+    with pytest.raises(binding.BpdqError) as ei:
+        binding.bpdq_pack(bits, np.zeros((3, 16, 1), dtype=np.uint16), 128)
+    assert ei.value.code == binding.ERR_INVALID and "bit value" in str(ei.value)
