@@ -59,6 +59,7 @@ extern "C" int bpdq_create(bpdq_handle_t* hp, int out, int in, int K, int group,
     std::memset(h, 0, sizeof(*h));
     h->out = out; h->in = in; h->K = K; h->group = group; h->max_M = max_M; h->device = dev;
     h->sm_count = prop.multiProcessorCount;
+    h->smem_optin = (int)prop.sharedMemPerBlockOptin;
     h->planes_bytes = planes_bytes(out, in, K);
     h->blob_bytes = h->planes_bytes + coefs_bytes(out, in, K, group);
     h->ws_bytes = gemv_workspace_bytes(out, in, K, group, max_M, h->sm_count);
@@ -78,6 +79,7 @@ extern "C" int bpdq_create(bpdq_handle_t* hp, int out, int in, int K, int group,
     }
     cudaMemset(h->d_counters, 0, (h->n_counters ? h->n_counters : 1) * sizeof(unsigned));
     cudaMemset(h->d_status, 0, sizeof(int));
+    cudaMemset(h->d_ws, 0, h->ws_bytes ? h->ws_bytes : 16);
     int rc = BPDQ_OK;
     if (host_blob) {
         e = cudaMemcpy(h->d_blob, host_blob, h->blob_bytes, cudaMemcpyHostToDevice);

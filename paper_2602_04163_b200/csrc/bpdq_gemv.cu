@@ -1,7 +1,450 @@
+// bpdq_gemv: batch-1 (M <= 2 per pass) evaluation of y = x * W^T straight from the packed planes.
+//
+// Method.  With Eq. 1 the dot product of a row with x regroups into the add-only form the paper
+// points to for bit-plane hardware and for its look-up-table decode kernel:
+//
+//     y[r] = sum_G ( c0[r,G] * X_G  +  sum_i ci[r,G] * S_i[r,G] ),
+//     X_G = sum of x over group G,    S_i[r,G] = sum of x_j over the set bits of plane i in G.
+//
+// S_i is read from look-up tables instead of being added bit by bit: for every 8 consecutive
+// inputs ("chunk") the 256 subset sums of x are precomputed in shared memory (binary32), so one
+// plane BYTE costs one byte-permute (address), one shared-memory load and one add.
+//
+// Work split.  A CTA owns a slice of 512 input columns (4 blocks of 128) and a range of 16-row
+// groups; it builds the 64 chunk tables of its slice once (64 KB per token) and then streams
+// planes.  A warp takes 16 rows x 4 blocks: lane (h, a) = (lane/16, lane%16) owns row a and the
+// two blocks of parity h; its 16-byte plane units and coefficients arrive through a per-warp
+// cp.async ring several tasks deep (HBM latency is covered by bytes in flight, not by registers),
+// and it walks the 16 bytes of each unit.  The blob stores byte p of row r as chunk (p + r) mod 16,
+// and table entries are laid out as [entry][slot], slot = 16*block + chunk, so at every step the
+// 32 lanes of a warp hit 32 different banks whatever the data: table loads are conflict-free by
+// construction.  The tables start at a multiple of 64 KB in the shared window, so the byte-permute
+// that splices the plane byte into bits 8..15 of the lane's slot address yields the final address.
+// Row sums are combined across slices with binary32 atomic adds into a small workspace
+// [token][row] that lives in L2; per 128 rows an arrival counter tells the CTA that delivers the
+// last contribution to round those rows to binary16, write y and zero the workspace again.
+// Algorithmic HBM bytes per weight: K/8 + 2(K+1)/g.
 #include "bpdq_internal.h"
-namespace bpdq {
-size_t gemv_workspace_bytes(int, int, int, int, int, int) { return 0; }
-size_t gemv_counter_count(int) { return 0; }
-bool gemv_supported(int, int, int, int) { return false; }
-int launch_gemv(bpdq_handle_s*, const void*, void*, int, cudaStream_t) { return set_error(BPDQ_ERR_UNSUPPORTED, "gemv: not built"); }
+
+#include <cuda_fp16.h>
+
+namespace {
+
+constexpr int kSliceBlocks = 4;                       // 128-column blocks per slice
+constexpr int kSlots = 16 * kSliceBlocks;             // chunk tables per slice = slots per entry row
+constexpr int kTableBytes = 256 * kSlots * 4;         // one token's tables: 64 KB
+constexpr int kMaxMT = 2;                             // tokens per pass (64 KB of tables each)
+constexpr int kChunkRgs = 8;                          // row groups (of 16 rows) per completion counter
+constexpr int kMaxStages = 8;                         // depth limit of a warp's staging ring
+constexpr int kMiscBytes = 4096;                      // xsum + completion list, at the start of shared memory
+constexpr int kMaxDone = 512;                         // completed chunks handled per batch
+
+struct GemvParams {
+    const uint8_t* blob;
+    size_t planes_bytes;
+    const __half* x;          // [MT][in]
+    __half* y;                // [MT][out]
+    float* ws;                // [MT][out] binary32 row sums, zero between calls
+    unsigned* counters;       // [ceil(out/16 / kChunkRgs)] arrival counters, zero between calls
+    int* status;              // device status word
+    int out, in, group;
+    int nblocks, nslices, nrg;
+    int tasks_base, tasks_rem;   // task range of CTA b: b*base + min(b, rem), one longer for b < rem
+    int dyn_smem;                // dynamic shared memory bytes of the launch
+};
+
+// One stage of a warp's staging ring holds one task (16 rows x 4 blocks): the lanes' plane units
+// ([q][plane][lane] x 16 bytes, each lane copies its own) and the task's coefficients
+// ([block][coefficient][row] binary16: 4(K+1) runs of 32 bytes, copied as 16-byte halves by the
+// first 8(K+1) lanes).  Coefficients are read by other lanes than copied them, so the warp
+// synchronises after its cp.async groups have landed.
+template <int K>
+struct Stage {
+    static constexpr int kPlaneBytes = 2 * K * 32 * 16;
+    static constexpr int kCoefSegs = kSliceBlocks * (K + 1);          // 32-byte runs per task
+    static constexpr int kCoefBytes = (kCoefSegs * 32 + 127) / 128 * 128;
+    static constexpr int kBytes = kPlaneBytes + kCoefBytes;
+};
+
+__device__ __forceinline__ void cp_async16(unsigned dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
+__device__ __forceinline__ void cp_async4(unsigned dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_dyn(int pending) {
+    switch (pending) {
+        case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+        case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+        case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+        case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+        case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+        case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
+        case 6: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
+    }
+}
+__device__ __forceinline__ uint4 lds_v4(unsigned addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ unsigned short lds_u16(unsigned addr) {
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+    return v;
+}
+// Table load.  Not volatile: its address is computed from plane bytes that were read after the
+// barrier that published the tables, so it cannot move above that barrier, and the compiler may
+// interleave the 32 independent look-ups of a plane unit freely.
+template <int IMM>
+__device__ __forceinline__ float lds_table(unsigned addr) {
+    float v;
+    asm("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"(IMM));
+    return v;
+}
+__device__ __forceinline__ unsigned word_of(const uint4& v, int k) {
+    return k == 0 ? v.x : k == 1 ? v.y : k == 2 ? v.z : v.w;
+}
+
+template <int K, int MT, int W>
+__global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p) {
+    constexpr int kThreads = W * 32;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int h = lane >> 4, a = lane & 15;
+
+    // ---- shared memory map (addresses in the shared window) ----
+    //   [smem0, +kMiscBytes)             xsum, completion list
+    //   [.., lut0)                       staging slots (low region)
+    //   [lut0, lut0 + MT*64 KB)          tables, lut0 a multiple of 64 KB
+    //   [.., smem0 + dyn_smem)           staging slots (high region)
+    const unsigned smem0 = (unsigned)__cvta_generic_to_shared(smem);
+    const unsigned lut0 = (smem0 + kMiscBytes + 65535u) & ~65535u;
+    const unsigned low0 = smem0 + kMiscBytes;
+    const int nlow = (int)(lut0 - low0) / Stage<K>::kBytes;
+    const unsigned high0 = lut0 + MT * kTableBytes;
+    const int nhigh = ((int)(smem0 + p.dyn_smem) - (int)high0) / Stage<K>::kBytes;
+    int stages = (nlow + (nhigh > 0 ? nhigh : 0)) / W;
+    if (stages > kMaxStages) stages = kMaxStages;
+    if ((int)(smem0 + p.dyn_smem) < (int)high0 || stages < 1) {   // tables or one slot per warp do not fit
+        if (tid == 0) atomicExch(p.status, BPDQ_ERR_UNSUPPORTED);
+        return;                                                    // uniform: no barrier has been reached
+    }
+    float* xsum = reinterpret_cast<float*>(smem);                         // [MT][kSliceBlocks]
+    int* done = reinterpret_cast<int*>(smem + 64);                        // [kMaxDone]
+    int* ndone = done + kMaxDone;
+    float* lut = reinterpret_cast<float*>(smem + (lut0 - smem0));         // [MT][256][kSlots]
+
+    // slot address of stage j of this warp
+    auto slot_addr = [&](int j) -> unsigned {
+        const int k = wid * stages + j;
+        return k < nlow ? low0 + k * Stage<K>::kBytes : high0 + (k - nlow) * Stage<K>::kBytes;
+    };
+
+    // the lane's table-slot address per step: lut0 + 4*((s + a) mod 16) + 64*h; the plane byte is
+    // spliced into bits 8..15 (entry row stride 256 B)
+    unsigned off[16];
+#pragma unroll
+    for (int s = 0; s < 16; ++s) off[s] = lut0 + 4u * ((s + a) & 15) + 64u * h;
+
+    // contiguous share of the (slice, row group) task space: base tasks each, the first `rem` CTAs one more
+    const int bid = blockIdx.x;
+    int t = bid * p.tasks_base + min(bid, p.tasks_rem);
+    const int t_end = t + p.tasks_base + (bid < p.tasks_rem ? 1 : 0);
+    const uint8_t* cbase = p.blob + p.planes_bytes;
+    const size_t plane_pitch = (size_t)p.out * 16;    // bytes between planes of one block
+
+    while (t < t_end) {
+        const int s = t / p.nrg;
+        const int rg_begin = t - s * p.nrg;
+        const int rg_end = min(p.nrg, rg_begin + (t_end - t));
+        const int ntask = (rg_end - rg_begin - wid + W - 1) / W;          // tasks of this warp (may be <= 0)
+
+        // per-lane source pointers of the first task; a task further on is W*16 rows further on
+        const uint8_t* psrc[2];
+        bool valid[2];
+        {
+            const int r = (rg_begin + wid) * 16 + a;
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int b = s * kSliceBlocks + 2 * q + h;
+                valid[q] = b < p.nblocks;
+                psrc[q] = p.blob + ((size_t)b * K * p.out + r) * 16;
+            }
+        }
+        // coefficient runs: copy slot L (one per lane, two rounds when 8(K+1) > 32) is half (L & 1)
+        // of run L >> 1 = (block, coefficient)
+        constexpr int kCoefRounds = (Stage<K>::kCoefSegs * 2 + 31) / 32;
+        const uint8_t* csrc[kCoefRounds];
+        int cstate[kCoefRounds];                      // 0: no copy, 1: copy, 2: zero-fill
+#pragma unroll
+        for (int c = 0; c < kCoefRounds; ++c) {
+            const int L = c * 32 + lane, seg = L >> 1;
+            const int blk = seg / (K + 1), i = seg - blk * (K + 1);
+            const int b = s * kSliceBlocks + blk;
+            const int G = (b * 128) / p.group;
+            cstate[c] = (seg >= Stage<K>::kCoefSegs) ? 0 : (b < p.nblocks ? 1 : 2);
+            csrc[c] = cbase + (((size_t)G * (K + 1) + i) * p.out + (size_t)(rg_begin + wid) * 16) * 2 + (L & 1) * 16;
+        }
+        auto issue_task = [&](int n, unsigned dst) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const unsigned pdst = dst + (q * K) * 512 + lane * 16;
+                if (valid[q]) {
+                    const uint8_t* ps = psrc[q] + (size_t)n * (W * 256);
+#pragma unroll
+                    for (int i = 0; i < K; ++i) cp_async16(pdst + i * 512, ps + i * plane_pitch);
+                } else {                              // block past the end of a ragged last slice
+#pragma unroll
+                    for (int i = 0; i < K; ++i)
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(pdst + i * 512), "r"(0u) : "memory");
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < kCoefRounds; ++c) {
+                const unsigned cdst = dst + Stage<K>::kPlaneBytes + (c * 32 + lane) * 16;
+                if (cstate[c] == 1) cp_async16(cdst, csrc[c] + (size_t)n * (W * 32));
+                else if (cstate[c] == 2)
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(cdst), "r"(0u) : "memory");
+            }
+        };
+
+        // the first tasks are requested before the tables are built, to overlap the latency
+        for (int n = 0; n < stages - 1; ++n) {
+            if (n < ntask) issue_task(n, slot_addr(n));
+            cp_async_commit();
+        }
+
+        // ---- build the 64 chunk tables of this slice (per token) ----
+        for (int item = tid; item < kSlots * 8; item += kThreads) {
+            const int slot = item & (kSlots - 1);     // chunk table
+            const int eh = item >> 6;                 // entries eh*32 .. eh*32+31 share inputs 5..7
+            const int col = s * (kSliceBlocks * 128) + slot * 8;
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                float xs[8];
+                if (col < p.in) {
+                    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(p.x + (size_t)m * p.in + col));
+                    const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float2 f = __half22float2(h2[k]);
+                        xs[2 * k] = f.x; xs[2 * k + 1] = f.y;
+                    }
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) xs[k] = 0.f;
+                }
+                float lo[32];                         // subset sums of inputs 0..4
+                lo[0] = 0.f;
+#pragma unroll
+                for (int k = 0; k < 5; ++k)
+#pragma unroll
+                    for (int j = 0; j < (1 << k); ++j) lo[(1 << k) + j] = lo[j] + xs[k];
+                float base = 0.f;
+                if (eh & 1) base += xs[5];
+                if (eh & 2) base += xs[6];
+                if (eh & 4) base += xs[7];
+                float* dst = lut + m * (kTableBytes / 4) + (eh * 32) * kSlots + slot;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) dst[j * kSlots] = base + lo[j];
+            }
+        }
+        __syncthreads();
+        if (tid < MT * kSliceBlocks) {
+            const int m = tid / kSliceBlocks, blk = tid % kSliceBlocks;
+            float acc = 0.f;
+            for (int c = 0; c < 16; ++c) acc += lut[m * (kTableBytes / 4) + 255 * kSlots + blk * 16 + c];
+            xsum[m * kSliceBlocks + blk] = acc;
+        }
+        __syncthreads();
+
+        // ---- stream the row groups of this slice ----
+        int stage_rd = 0, stage_wr = stages - 1;
+        for (int n = 0; n < ntask; ++n) {
+            {
+                const int nn = n + stages - 1;
+                if (nn < ntask) issue_task(nn, slot_addr(stage_wr));
+                cp_async_commit();
+                stage_wr = (stage_wr + 1 == stages) ? 0 : stage_wr + 1;
+            }
+            cp_async_wait_dyn(stages - 1);            // all but the newest stages-1 groups are complete: task n has landed
+            __syncwarp();                             // ... for every lane: coefficients are read across lanes
+            const unsigned st_base = slot_addr(stage_rd);
+            stage_rd = (stage_rd + 1 == stages) ? 0 : stage_rd + 1;
+
+            float yacc[MT];
+#pragma unroll
+            for (int m = 0; m < MT; ++m) yacc[m] = 0.f;
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                float S[K][MT][2];                    // two partial sums per plane shorten the add chains
+                uint4 pl[K];
+#pragma unroll
+                for (int i = 0; i < K; ++i) {
+                    pl[i] = lds_v4(st_base + (q * K + i) * 512 + lane * 16);
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) S[i][m][0] = S[i][m][1] = 0.f;
+                }
+#pragma unroll
+                for (int st = 0; st < 16; ++st) {
+#pragma unroll
+                    for (int i = 0; i < K; ++i) {
+                        // address = slot address with the plane byte in bits 8..15
+                        const unsigned addr = __byte_perm(word_of(pl[i], st >> 2), off[st], 0x7604u | ((st & 3) << 4));
+#pragma unroll
+                        for (int m = 0; m < MT; ++m) {      // the token's table and the block pair go into the immediate
+                            if (m == 0 && q == 0) S[i][m][st & 1] += lds_table<0>(addr);
+                            else if (m == 0) S[i][m][st & 1] += lds_table<128>(addr);
+                            else if (q == 0) S[i][m][st & 1] += lds_table<kTableBytes>(addr);
+                            else S[i][m][st & 1] += lds_table<kTableBytes + 128>(addr);
+                        }
+                    }
+                }
+                const int blk = 2 * q + h;
+                const unsigned cw = st_base + Stage<K>::kPlaneBytes + (blk * (K + 1)) * 32 + a * 2;
+                const float c0 = __half2float(__ushort_as_half(lds_u16(cw)));
+#pragma unroll
+                for (int m = 0; m < MT; ++m) yacc[m] = fmaf(c0, xsum[m * kSliceBlocks + blk], yacc[m]);
+#pragma unroll
+                for (int i = 0; i < K; ++i) {
+                    const float ci = __half2float(__ushort_as_half(lds_u16(cw + (i + 1) * 32)));
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) yacc[m] = fmaf(ci, S[i][m][0] + S[i][m][1], yacc[m]);
+                }
+            }
+            __syncwarp();                             // the stage is refilled by the next iteration's copies
+            // the two half-warps hold the even-block and odd-block parts of the same 16 rows
+#pragma unroll
+            for (int m = 0; m < MT; ++m) yacc[m] += __shfl_xor_sync(0xffffffffu, yacc[m], 16);
+            if (h == 0) {
+                const int r = (rg_begin + wid + n * W) * 16 + a;
+#pragma unroll
+                for (int m = 0; m < MT; ++m) atomicAdd(&p.ws[(size_t)m * p.out + r], yacc[m]);
+            }
+        }
+        cp_async_wait_dyn(0);
+
+        // ---- hand this segment over ----
+        // Row sums are accumulated across slices with binary32 atomic adds in `ws` (kept zero
+        // between calls).  Row groups are counted in chunks of kChunkRgs; whoever delivers the last
+        // contribution of a chunk converts its rows to binary16, writes y and zeroes `ws` again.
+        __threadfence();
+        __syncthreads();
+        const int ck_begin = rg_begin / kChunkRgs, ck_end = (rg_end + kChunkRgs - 1) / kChunkRgs;
+        for (int ck0 = ck_begin; ck0 < ck_end; ck0 += kMaxDone) {
+            if (tid == 0) *ndone = 0;
+            __syncthreads();
+            for (int ck = ck0 + tid; ck < min(ck_end, ck0 + kMaxDone); ck += kThreads) {
+                const int lo = max(rg_begin, ck * kChunkRgs), hi = min(rg_end, (ck + 1) * kChunkRgs);
+                const int size = min(p.nrg, (ck + 1) * kChunkRgs) - ck * kChunkRgs;
+                const unsigned before = atomicAdd(&p.counters[ck], (unsigned)(hi - lo));
+                if (before + (unsigned)(hi - lo) == (unsigned)(size * p.nslices)) {
+                    p.counters[ck] = 0u;
+                    done[atomicAdd(ndone, 1)] = ck;
+                }
+            }
+            __syncthreads();
+            const int nd = *ndone;
+            if (nd > 0) {
+                __threadfence();
+                for (int idx = tid; idx < nd * kChunkRgs * 16 * MT; idx += kThreads) {
+                    const int ckd = done[idx / (kChunkRgs * 16 * MT)];
+                    const int rem = idx % (kChunkRgs * 16 * MT);
+                    const int m = rem / (kChunkRgs * 16);
+                    const int r = ckd * kChunkRgs * 16 + rem % (kChunkRgs * 16);
+                    if (r < p.out) {
+                        float* src = p.ws + (size_t)m * p.out + r;
+                        p.y[(size_t)m * p.out + r] = __float2half_rn(__ldcg(src));
+                        __stcg(src, 0.f);
+                    }
+                }
+            }
+            __syncthreads();
+        }
+        t += rg_end - rg_begin;
+    }
+}
+
+template <int K, int MT, int W>
+int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
+    static int configured_smem = 0;
+    const int smem = h->smem_optin;
+    if (configured_smem != smem) {
+        cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<K, MT, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemv: shared memory opt-in: %s", cudaGetErrorString(e));
+        configured_smem = smem;
+    }
+    const long long total = (long long)p.nslices * p.nrg;
+    if (total >= (1ll << 31)) return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv: task space too large");
+    int grid = h->sm_count;
+    if ((long long)grid > total) grid = (int)total;
+    p.tasks_base = (int)(total / grid);
+    p.tasks_rem = (int)(total % grid);
+    p.dyn_smem = smem;
+    gemv_lut_kernel<K, MT, W><<<grid, W * 32, smem, stream>>>(p);
+    h->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemv launch: %s", cudaGetErrorString(e));
+    return BPDQ_OK;
+}
+
+// Warps per CTA: 16 when at least two ring stages per warp fit beside the tables, else 8.
+template <int K, int MT>
+int launch_one(bpdq_handle_s* h, const GemvParams& p, cudaStream_t stream) {
+    const int ring_bytes = h->smem_optin - 2048 - kMiscBytes - MT * kTableBytes;   // 2 KB: allowance for the window base
+    if (ring_bytes / (16 * Stage<K>::kBytes) >= 2) return launch_cfg<K, MT, 16>(h, p, stream);
+    if (ring_bytes / (8 * Stage<K>::kBytes) >= 1) return launch_cfg<K, MT, 8>(h, p, stream);
+    return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv: staging ring does not fit (K=%d, tokens=%d)", K, MT);
+}
+
+template <int K>
+int launch_k(bpdq_handle_s* h, GemvParams p, const __half* x, __half* y, int M, cudaStream_t stream) {
+    int m0 = 0;
+    while (m0 < M) {
+        int mt = M - m0;
+        if (mt > kMaxMT) mt = kMaxMT;
+        p.x = x + (size_t)m0 * h->in;
+        p.y = y + (size_t)m0 * h->out;
+        const int rc = (mt == 1) ? launch_one<K, 1>(h, p, stream) : launch_one<K, 2>(h, p, stream);
+        if (rc != BPDQ_OK) return rc;
+        m0 += mt;
+    }
+    return BPDQ_OK;
+}
+
+}  // namespace
+
+namespace bpdq {
+
+bool gemv_supported(int, int, int K, int group) { return K >= 1 && K <= 4 && (group == 128 || group == 256); }
+
+size_t gemv_workspace_bytes(int out, int, int, int, int, int) { return kMaxMT * (size_t)out * sizeof(float); }
+
+size_t gemv_counter_count(int out) { return ((size_t)out / 16 + kChunkRgs - 1) / kChunkRgs; }
+
+int launch_gemv(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
+    GemvParams p;
+    p.blob = h->d_blob;
+    p.planes_bytes = h->planes_bytes;
+    p.ws = h->d_ws;
+    p.counters = h->d_counters;
+    p.status = h->d_status;
+    p.out = h->out; p.in = h->in; p.group = h->group;
+    p.nblocks = h->in / 128;
+    p.nslices = (p.nblocks + kSliceBlocks - 1) / kSliceBlocks;
+    p.nrg = h->out / 16;
+    const __half* xp = static_cast<const __half*>(x);
+    __half* yp = static_cast<__half*>(y);
+    switch (h->K) {
+        case 1: return launch_k<1>(h, p, xp, yp, M, stream);
+        case 2: return launch_k<2>(h, p, xp, yp, M, stream);
+        case 3: return launch_k<3>(h, p, xp, yp, M, stream);
+        case 4: return launch_k<4>(h, p, xp, yp, M, stream);
+        default: return set_error(BPDQ_ERR_UNSUPPORTED, "gemv: K=%d", h->K);
+    }
+}
+
+}  // namespace bpdq

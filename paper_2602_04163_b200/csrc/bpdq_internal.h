@@ -38,11 +38,12 @@ int set_error(int code, const char* fmt, ...);
 struct bpdq_handle_s {
     int out, in, K, group, max_M, device;
     int sm_count;
+    int smem_optin;           // largest dynamic shared memory a CTA may opt in to
     uint8_t* d_blob;          // planes then coefficients
     size_t blob_bytes, planes_bytes;
-    float* d_ws;              // split-K partial sums
+    float* d_ws;              // binary32 row sums of the split over input slices (zero between calls)
     size_t ws_bytes;
-    unsigned* d_counters;     // one arrival counter per 32-row block (self-resetting)
+    unsigned* d_counters;     // arrival counters per 128 rows (zero between calls)
     size_t n_counters;
     int* d_status;            // device status word
     void* d_xstage;           // staging for bpdq_linear_host

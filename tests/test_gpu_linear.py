@@ -32,3 +32,66 @@ def test_m_zero_and_bad_arguments():
     with pytest.raises(binding.BpdqError):
         h.bpdq_linear_ex(x.data_ptr(), y.data_ptr(), 1, 99, G.stream_ptr())
     assert h.bpdq_launch_count() == n0                                   # no launch on rejected calls
+
+
+@pytest.mark.parametrize("K,g,out,in_,M", [
+    (2, 128, 160, 640, 1),       # 5 blocks: the second slice is ragged (1 block)
+    (3, 128, 96, 384, 1),        # 3 blocks: a single ragged slice
+    (2, 128, 4096, 4096, 1),     # benchmark config 1
+    (3, 128, 1024, 2048, 2),
+    (2, 256, 64, 1024, 3),
+    (1, 128, 32, 128, 1),
+    (4, 128, 48, 1536, 2),
+    (2, 128, 272, 896, 4),       # 4 tokens = two passes of 2
+    (3, 128, 144, 512, 7),       # 3 + 2 + 2
+    (2, 128, 16, 128, 1),        # smallest supported shape
+])
+def test_lut_kernel(K, g, out, in_, M):
+    h, bits, coef = G.make_layer(40 + K, out, in_, K, g, max_M=M)
+    x = synth.activations(50 + K, M, in_)
+    rows = None
+    if out * in_ > 2 ** 22:      # keep the checker's share to seconds: sampled rows, every tile boundary
+        rows = np.unique(np.concatenate([np.arange(0, out, 61), [15, 16, 31, 32, out - 17, out - 16, out - 1]]))
+    G.check_linear(h, bits, coef, x, g, binding.KERNEL_GEMV, rows=rows, what="lut")
+    # slices are combined with binary32 atomic adds whose order is free: two calls may differ by
+    # the last binary16 digit, no more (and the workspace must come back clean for the second call)
+    y1 = G.run_linear(h, x, binding.KERNEL_GEMV)
+    y2 = G.run_linear(h, x, binding.KERNEL_GEMV)
+    assert np.allclose(y1, y2, rtol=2.0 ** -9, atol=1e-5)
+    # and the cross-check kernel agrees to within the same bound
+    y3 = G.run_linear(h, x, binding.KERNEL_GEMV_SIMPLE)
+    assert np.max(np.abs(y1 - y3)) <= 0.05 + 0.01 * np.max(np.abs(y3))
+
+
+def test_lut_kernel_special_inputs():
+    """All-zero planes (y = sum_G c0 X_G), all-one planes, one-hot activations."""
+    K, g, out, in_ = 2, 128, 64, 1024
+    coef = synth.coefficients(8, out, in_, K, g)
+    x = synth.activations(8, 1, in_)
+    for fill in (0, 1):
+        bits = np.full((K, out, in_), fill, dtype=np.uint8)
+        h = binding.Handle(out, in_, K, g, binding.bpdq_pack(bits, coef, g), 0, 1)
+        G.check_linear(h, bits, coef, x, g, binding.KERNEL_GEMV, what=f"fill{fill}")
+    bits = synth.plane_bits(8, out, in_, K)
+    h = binding.Handle(out, in_, K, g, binding.bpdq_pack(bits, coef, g), 0, 1)
+    w = oracle.dequant(bits, coef, g).view(np.float16).astype(np.float64)
+    for j in (0, 7, 8, 127, 128, 511, 512, 1023):
+        xo = np.zeros((1, in_), dtype=np.float16)
+        xo[0, j] = 1.0
+        y = G.run_linear(h, xo.view(np.uint16), binding.KERNEL_GEMV)
+        assert np.max(np.abs(y[0] - w[:, j])) <= 2.0 ** -10 * np.max(np.abs(w[:, j])) + 1e-6, j
+
+
+@pytest.mark.parametrize("name,out,in_,K", [("gate", 29568, 8192, 2), ("down", 8192, 29568, 3), ("k", 1024, 8192, 2),
+                                             ("7b_down", 3584, 18944, 2)])
+def test_lut_kernel_full_size_sampled(name, out, in_, K):
+    """Benchmark-sized layers generated on the device; sampled rows against the checker."""
+    g = 128
+    h = binding.Handle(out, in_, K, g, None, 900 + K, 1)
+    x = synth.activations(901, 1, in_)
+    y = G.run_linear(h, x, binding.KERNEL_GEMV)
+    rows = np.unique(np.concatenate([np.arange(0, out, max(1, out // 40)), [0, 15, 16, out - 16, out - 1]]))
+    y_ref, a_ref = oracle.linear(synth.plane_bits(900 + K, out, in_, K, rows),
+                                 synth.coefficients(900 + K, out, in_, K, g, rows), x, g)
+    G.assert_linear_close(y[:, rows], y_ref, a_ref, name)
+    assert np.all(np.isfinite(y))
