@@ -1,0 +1,378 @@
+"""Benchmark of the BPDQ weight-only linear layer (decode GEMV, prefill GEMM, dequant) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-extras]
+
+One JSON line on stdout.  The headline workload is a Qwen2.5-72B-shaped decoder layer at K = 2
+bit-planes, group 128, one token (M = 1): a step is one pass of bpdq_linear over the layer's seven
+linears.  Several distinct copies of the layer are rotated between steps so that no weight byte can
+be served from L2.  `value` is the useful HBM bytes (packed planes + coefficients + x + y) moved per
+second; the `roofline` object relates it to the measured copy bandwidth.  Further timed sections
+(K = 3 layer, fused qkv / gate-up handles, prefill GEMM, dequant) are reported under `sections`.
+
+With --gpus N > 1 (launched under torchrun) every rank runs an independent replica of the same
+workload ("replicas only": the path has no exchange step); the value is the sum over ranks divided
+by the slowest rank's time.
+
+--impl reference times the plain C++ checker under oracle/ on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2602_04163_b200 import synth  # noqa: E402
+
+METRIC = "bpdq_gemv_useful_hbm_gbs_batch1_72b_layer"
+UNIT = "GB/s"
+GROUP = 128
+HBM_NOMINAL_GBS = 8000.0
+FALLBACK_HBM_GBS, FALLBACK_TFLOPS = 6650.0, 1590.0
+
+
+def useful_bytes(out: int, in_: int, K: int, g: int, M: int) -> int:
+    """Algorithmic HBM bytes of one linear call: packed planes + binary16 coefficients + x + y."""
+    return out * in_ * K // 8 + out * (in_ // g) * (K + 1) * 2 + M * in_ * 2 + M * out * 2
+
+
+def layer_bytes(shapes, K: int, M: int) -> int:
+    return sum(useful_bytes(o, i, K, GROUP, M) for _, o, i in shapes)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "tflops": float(d["bf16_tflops"]),
+                "tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "tflops": FALLBACK_TFLOPS, "tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc, self.thread = index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = [r for t, r in self.rows if t0 <= t <= t1 + 0.2 and len(r) >= 7] or [r for _, r in self.rows if len(r) >= 7]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = sorted(float(r[0]) for r in rows)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for k, n in enumerate(names) if any(r[3 + k].lower().startswith("active") for r in rows)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(rows[0][1]), "reasons": reasons,
+                "samples": len(rows), "power_w_max": max(float(r[2]) for r in rows)}
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm: the checker under oracle/, as it stands, on the host cores
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(shapes, K: int, rows_per_linear: int, seed: int = 0):
+    """Logical tensors of `rows_per_linear` evenly spaced output rows of every linear of the layer."""
+    sample = []
+    for li, (name, out, in_) in enumerate(shapes):
+        s = synth.linear_seed(seed, 0, li, K)
+        rows = np.unique(np.linspace(0, out - 1, rows_per_linear).astype(np.int64))
+        sample.append((name, out, in_, synth.plane_bits(s, out, in_, K, rows),
+                       synth.coefficients(s, out, in_, K, GROUP, rows), synth.activations(s + 1, 1, in_)))
+    return sample
+
+
+def time_oracle(sample, K: int):
+    """Runs the checker's linear map over the sample once; returns (seconds, useful bytes covered)."""
+    import oracle
+    covered = 0
+    t0 = time.perf_counter()
+    for _, out, in_, bits, coef, x in sample:
+        oracle.linear(bits, coef, x, GROUP)
+        n = bits.shape[1]
+        covered += useful_bytes(n, in_, K, GROUP, 1)
+    return time.perf_counter() - t0, covered
+
+
+def run_reference(args, rank: int):
+    if rank != 0:
+        return
+    shapes, K = synth.QWEN25_72B_LAYER, 2
+    # bounded sample: the whole run (warm-up included) stays near one minute at the checker's ~8e6 weights/s
+    cols = sum(i for _, _, i in shapes)
+    rows = max(2, min(512, int(60.0 * 8e6 / (cols * max(1, args.steps + args.warmup)))))
+    sample = oracle_sample(shapes, K, rows)
+    import oracle
+    oracle.build()
+    for _ in range(args.warmup):
+        time_oracle(sample, K)
+    t_total, covered = 0.0, 0
+    for _ in range(args.steps):
+        dt, nb = time_oracle(sample, K)
+        t_total += dt
+        covered += nb
+    value = covered / t_total / 1e9
+    desc = f"{rows} evenly spaced output rows of each of the 7 linears per step, single thread"
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "impl": "reference", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "qwen2.5-72b-shaped decoder layer, K=2, g=128, M=1 (7 linears)", "sample": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# CUDA arm
+# ------------------------------------------------------------------------------------------------
+class Layer:
+    """Handles of one decoder layer's linears, generated on the device from a seed."""
+
+    def __init__(self, shapes, K: int, seed: int, layer: int, max_M: int):
+        from paper_2602_04163_b200 import binding
+        self.handles = []
+        for li, (name, out, in_) in enumerate(shapes):
+            self.handles.append((name, binding.Handle(out, in_, K, GROUP, None, synth.linear_seed(seed, layer, li, K), max_M)))
+
+    def destroy(self):
+        for _, h in self.handles:
+            h.bpdq_destroy()
+
+
+def event_time_ms(torch, fn, stream):
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    fn()
+    e1.record(stream)
+    e1.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def run_cuda(args, rank: int, world: int, local_rank: int):
+    import torch
+    import torch.distributed as dist
+    from paper_2602_04163_b200 import binding
+
+    binding.lib()                      # raises if the CUDA library is missing: there is no other path
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+    peaks = measured_peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    shapes, K, M = synth.QWEN25_72B_LAYER, 2, 1
+    copies = 4
+    layers = [Layer(shapes, K, 0, c, 1) for c in range(copies)]
+    xs = {in_: torch.from_numpy(synth.activations(7, 1, in_).view(np.int16).copy()).cuda().view(torch.float16)
+          for in_ in sorted({i for _, _, i in shapes})}
+    ys = {out: torch.empty((1, out), dtype=torch.float16, device="cuda") for out in sorted({o for _, o, _ in shapes})}
+
+    def step(layer):
+        for (name, h) in layer.handles:
+            h.bpdq_linear(xs[h.in_].data_ptr(), ys[h.out].data_ptr(), M, sp)
+
+    launches0 = sum(h.bpdq_launch_count() for L in layers for _, h in L.handles)
+    for w in range(args.warmup):
+        step(layers[w % copies])
+    barrier()
+    launches1 = sum(h.bpdq_launch_count() for L in layers for _, h in L.handles)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    t_wall0 = time.time()
+    # the timed region: exactly `steps` steps, CUDA events on the launching stream
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for s in range(args.steps):
+        step(layers[s % copies])
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    t_wall1 = time.time()
+    launches2 = sum(h.bpdq_launch_count() for L in layers for _, h in L.handles)
+
+    # the timed region is microseconds long at small step counts; keep the GPU under the same load a
+    # little longer so that nvidia-smi (100 ms period) sees the clocks it ran at
+    t_hold = time.time()
+    while time.time() - t_hold < 1.0:
+        for s in range(50):
+            step(layers[s % copies])
+        torch.cuda.synchronize()
+    clocks = sampler.stop(t_wall0, time.time())
+
+    # end to end: x in pinned host memory, y back to pinned host memory, every step, through the C ABI
+    xh = {in_: torch.from_numpy(synth.activations(7, 1, in_).view(np.int16).copy()).view(torch.float16).pin_memory()
+          for in_ in xs}
+    yh = {out: torch.empty((1, out), dtype=torch.float16).pin_memory() for out in ys}
+
+    def step_host(layer):
+        for (name, h) in layer.handles:
+            h.bpdq_linear_host(xh[h.in_].data_ptr(), yh[h.out].data_ptr(), M, sp)
+
+    for w in range(max(3, args.warmup)):
+        step_host(layers[w % copies])
+    barrier()
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        step_host(layers[s % copies])
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+
+    times = torch.tensor([ms_total, e2e_s * 1e3], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = float(times[0]), float(times[1])
+    bytes_step = layer_bytes(shapes, K, M)
+    value = world * bytes_step * args.steps / (ms_total * 1e-3) / 1e9
+    e2e_value = world * bytes_step * args.steps / (e2e_ms * 1e-3) / 1e9
+    per_gpu = value / world
+    n_launch = (launches2 - launches1)
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "qwen2.5-72b-shaped decoder layer, K=2, g=128, M=1 (7 linears: q k v o gate up down)",
+                       "l2": f"inputs larger than L2: {copies} distinct layer copies of {bytes_step / 1e6:.1f} MB rotated between steps",
+                       "useful_bytes_per_step": bytes_step, "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "e2e": {"value": e2e_value, "unit": UNIT,
+                    "h2d_bytes_per_step": sum(2 * M * i for _, _, i in shapes), "d2h_bytes_per_step": sum(2 * M * o for _, o, _ in shapes)},
+            "gpu_launches": n_launch, "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": "gemv_lut_kernel", "achieved": per_gpu, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": per_gpu / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                         "frac_of_nominal_8tbs": per_gpu / HBM_NOMINAL_GBS, "traffic": None,
+                         "launches_per_step": len(shapes), "algorithmic_bytes_per_launch_avg": bytes_step / len(shapes)}}
+
+    if rank == 0 and not args.no_extras:
+        line["sections"] = extra_sections(torch, binding, args, peaks, sp, stream)
+    for L in layers:
+        L.destroy()
+
+    if rank == 0:
+        if world == 1:
+            line["cpu_baseline"] = cpu_baseline(shapes, K)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def cpu_baseline(shapes, K):
+    """The checker as it stands, single thread, on a bounded sample of the same layer (about 15 s)."""
+    import oracle
+    oracle.build()
+    rows = 1536
+    sample = oracle_sample(shapes, K, rows)
+    dt, covered = time_oracle(sample, K)
+    return {"value": covered / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
+            "sample": f"{rows} evenly spaced output rows of each of the 7 linears of the layer (M=1), one pass"}
+
+
+def extra_sections(torch, binding, args, peaks, sp, stream):
+    """Per-linear GEMV at K=2 and K=3, fused handles, dequant and the prefill GEMM, each timed alone."""
+    out = {}
+    steps = max(5, min(args.steps, 20))
+    l2_flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def timed(fn, n=steps):
+        ts = []
+        for _ in range(3):
+            fn()
+        for _ in range(n):
+            l2_flush.zero_()
+            ts.append(event_time_ms(torch, fn, stream))
+        ts.sort()
+        return ts[len(ts) // 2], ts[0]
+
+    shapes72 = synth.QWEN25_72B_LAYER
+    per_linear = []
+    cases = [("q/o", 8192, 8192), ("k/v", 1024, 8192), ("gate/up", 29568, 8192), ("down", 8192, 29568),
+             ("qkv fused", 10240, 8192), ("gate+up fused", 59136, 8192)]
+    for K in (2, 3):
+        for name, o, i in cases:
+            h = binding.Handle(o, i, K, GROUP, None, 11, 1)
+            x = torch.from_numpy(synth.activations(3, 1, i).view(np.int16).copy()).cuda().view(torch.float16)
+            y = torch.empty((1, o), dtype=torch.float16, device="cuda")
+            med, best = timed(lambda: h.bpdq_linear(x.data_ptr(), y.data_ptr(), 1, sp))
+            b = useful_bytes(o, i, K, GROUP, 1)
+            per_linear.append({"linear": name, "out": o, "in": i, "K": K, "us_median": med * 1e3, "us_best": best * 1e3,
+                               "gbs": b / (med * 1e-3) / 1e9, "frac_measured": b / (med * 1e-3) / 1e9 / peaks["hbm_gbs"]})
+            h.bpdq_destroy()
+    out["gemv_per_linear_l2_flushed"] = per_linear
+
+    # dequant of the gate projection
+    for K in (2, 3):
+        o, i = 29568, 8192
+        h = binding.Handle(o, i, K, GROUP, None, 12, 1)
+        w = torch.empty((o, i), dtype=torch.float16, device="cuda")
+        med, best = timed(lambda: h.bpdq_dequant(w.data_ptr(), sp), 5)
+        b = h.packed_bytes + o * i * 2
+        out[f"dequant_gate_K{K}"] = {"ms_median": med, "gbs": b / (med * 1e-3) / 1e9,
+                                     "frac_measured": b / (med * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        h.bpdq_destroy()
+        del w
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-extras", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+    run_cuda(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()
