@@ -40,8 +40,13 @@
  *            the units of consecutive rows are adjacent, so that a warp reads 32 rows with one
  *            coalesced 512-byte request and a 128-row tile is one contiguous 2 KB run:
  *              unit(b, i, r) at byte ((b*K + i)*out + r)*16,   b = floor(j/128), i 0-based.
- *            Inside a unit the sixteen 8-column bytes are rotated by the row number: byte p
- *            holds columns 128*b + 8*((p + r) mod 16) + t, bit t (LSB = 0).  Rows that a
+ *            Inside a unit: word k (k = 0..3, little-endian bytes 4k..4k+3) covers columns
+ *            128*b + 32*k .. + 31, and bit 4*j + u of that word is column 128*b + 32*k + 8*u + j
+ *            (j = 0..7, u = 0..3): eight consecutive columns sit one bit per nibble, which is the
+ *            form the tensor-core kernel's byte-permute decode consumes.  Byte q of word k
+ *            ("logical byte" L = 4*k + q) therefore holds, at bit 4*jj + u, column
+ *            128*b + 32*k + 8*u + 2*q + jj (jj = 0..1).  The sixteen bytes are then rotated by
+ *            the row number: physical byte p holds logical byte (p + r) mod 16.  Rows that a
  *            half-warp handles together therefore index sixteen different 8-column look-up
  *            tables at every step.
  *   coefs  : binary16 at byte planes_bytes + ((G*(K+1) + i)*out + r)*2.

@@ -33,8 +33,9 @@
 // oracle_unpack is an independent reader of the device blob layout, written from the
 // layout's description (not from the library's packer):
 //   planes : for block b = floor(j/128), plane i (0-based), row r: 16 bytes at byte offset
-//            ((b*K + i)*out + r)*16;  byte p of that unit holds the 8 columns
-//            128*b + 8*((p + r) mod 16) + t, t = bit number (LSB = 0);
+//            ((b*K + i)*out + r)*16;  byte p of that unit is "logical byte" L = (p + r) mod 16,
+//            which belongs to 32-column word k = L / 4 as its byte q = L % 4; bit t of the byte
+//            (LSB = 0), split as t = 4*jj + u, is column 128*b + 32*k + 8*u + 2*q + jj;
 //   coefs  : after all planes; fp16 at byte offset ((G*(K+1) + i)*out + r)*2, i = 0 is c0.
 #include <cmath>
 #include <cstdint>
@@ -167,10 +168,13 @@ int oracle_unpack(const uint8_t* blob, int64_t out, int64_t in, int K, int64_t g
             for (int64_t r = 0; r < out; ++r) {
                 const uint8_t* unit = blob + ((b * K + i) * out + r) * 16;
                 for (int p = 0; p < 16; ++p) {
-                    const int64_t chunk = (p + r) % 16;
-                    for (int t = 0; t < 8; ++t)
-                        bits[((int64_t)i * out + r) * in + 128 * b + 8 * chunk + t] =
+                    const int64_t L = (p + r) % 16;
+                    const int64_t k = L / 4, q = L % 4;
+                    for (int t = 0; t < 8; ++t) {
+                        const int jj = t / 4, u = t % 4;
+                        bits[((int64_t)i * out + r) * in + 128 * b + 32 * k + 8 * u + 2 * q + jj] =
                             (uint8_t)((unit[p] >> t) & 1);
+                    }
                 }
             }
     const uint8_t* cbase = blob + out * in * K / 8;

@@ -5,9 +5,10 @@
 // builds the 2^K candidate values of its (row, group) (Eq. 7) with the decode rule's exact
 // arithmetic: float(c0), then "+ float(ci)" in binary32 for the set bits in plane order, one
 // rounding to binary16.  Units and candidate tables are staged in shared memory; the warp then
-// writes two rows per step, 16 lanes x 16 bytes each, so every row segment leaves as one
+// writes two rows per step, 16 lanes x 16 bytes each (eight consecutive columns: one bit per nibble of a logical word), so every row segment leaves as one
 // contiguous 256-byte store.  HBM-bound on the 2 bytes per weight it writes.
 #include "bpdq_internal.h"
+#include "bpdq_decode.cuh"
 
 #include <cuda_fp16.h>
 
@@ -39,7 +40,7 @@ dequant_kernel(const uint8_t* __restrict__ blob, size_t planes_bytes, __half* __
 #pragma unroll
             for (int i = 0; i < K; ++i) {
                 const uint4 u = *reinterpret_cast<const uint4*>(blob + bpdq::plane_unit_offset(b, i, r, K, out));
-                *reinterpret_cast<uint4*>(&s_units[wid][i][lane][0]) = u;
+                *reinterpret_cast<uint4*>(&s_units[wid][i][lane][0]) = bpdq::unrotate_unit(u, r);   // staged in logical byte order
             }
             for (int sub = 0; sub < nsub; ++sub) {
                 const int G = (b * 128 + sub * 64) / group;
@@ -65,16 +66,17 @@ dequant_kernel(const uint8_t* __restrict__ blob, size_t planes_bytes, __half* __
             const int lr = it * 2 + (lane >> 4);     // local row
             const int rr = rb * 32 + lr;
             if (rr < out) {
-                const int p = (c8 - rr) & 15;        // byte p holds chunk (p + row) mod 16
-                unsigned byte[K];
+                // columns 8*c8 .. 8*c8+7 are bits 4*t + u of logical word k, k = c8 / 4, u = c8 % 4
+                unsigned word[K];
 #pragma unroll
-                for (int i = 0; i < K; ++i) byte[i] = s_units[wid][i][lr][p];
+                for (int i = 0; i < K; ++i)
+                    word[i] = *reinterpret_cast<const unsigned*>(&s_units[wid][i][lr][(c8 >> 2) * 4]) >> (c8 & 3);
                 __align__(16) __half v[8];
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {
                     unsigned code = 0;
 #pragma unroll
-                    for (int i = 0; i < K; ++i) code |= ((byte[i] >> t) & 1u) << i;
+                    for (int i = 0; i < K; ++i) code |= ((word[i] >> (4 * t)) & 1u) << i;
                     v[t] = s_table[wid][lr][sub][code];
                 }
                 *reinterpret_cast<uint4*>(w + (size_t)rr * in + (size_t)b * 128 + c8 * 8) =

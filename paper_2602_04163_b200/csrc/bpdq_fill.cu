@@ -37,7 +37,18 @@ __global__ void fill_planes_kernel(uint8_t* __restrict__ blob, unsigned long lon
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const unsigned long long q = ((unsigned long long)i * out + r) * (unsigned long long)(in / 32) + 4ull * b + k;
-            logical[k] = (unsigned)(draw64(key, q) >> 32);
+            const unsigned drawn = (unsigned)(draw64(key, q) >> 32);       // bit t = column 32k + t
+            // layout word: bit 4j + u = column 32k + 8u + j, i.e. the bits of byte u spread one per nibble
+            unsigned word = 0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                unsigned x = (drawn >> (8 * u)) & 0xFFu;
+                x = (x | (x << 12)) & 0x000F000Fu;
+                x = (x | (x << 6)) & 0x03030303u;
+                x = (x | (x << 3)) & 0x11111111u;
+                word |= x << u;
+            }
+            logical[k] = word;
         }
         // physical byte p = logical byte (p + r) mod 16: rotate the 128-bit unit right by 8*(r mod 16) bits
         const int rot = (int)(r & 15);

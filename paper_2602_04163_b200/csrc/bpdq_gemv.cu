@@ -15,7 +15,7 @@
 // planes.  A warp takes 16 rows x 4 blocks: lane (h, a) = (lane/16, lane%16) owns row a and the
 // two blocks of parity h; its 16-byte plane units and coefficients arrive through a per-warp
 // cp.async ring several tasks deep (HBM latency is covered by bytes in flight, not by registers),
-// and it walks the 16 bytes of each unit.  The blob stores byte p of row r as chunk (p + r) mod 16,
+// and it walks the 16 bytes of each unit.  The blob stores, at byte p of row r, the 8-column chunk ("logical byte") (p + r) mod 16,
 // and table entries are laid out as [entry][slot], slot = 16*block + chunk, so at every step the
 // 32 lanes of a warp hit 32 different banks whatever the data: table loads are conflict-free by
 // construction.  The tables start at a multiple of 64 KB in the shared window, so the byte-permute
@@ -221,17 +221,18 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
         for (int item = tid; item < kSlots * 8; item += kThreads) {
             const int slot = item & (kSlots - 1);     // chunk table
             const int eh = item >> 6;                 // entries eh*32 .. eh*32+31 share inputs 5..7
-            const int col = s * (kSliceBlocks * 128) + slot * 8;
+            // slot = 16*block + logical byte L; L = 4k + q is byte q of 32-column word k, and bit
+            // 4*jj + u of that byte is column 32k + 8u + 2q + jj: four pairs of adjacent inputs
+            const int col = s * (kSliceBlocks * 128) + (slot >> 2) * 32 + (slot & 3) * 2;
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
-                float xs[8];
+                float xs[8];                          // xs[t]: the input that bit t of the plane byte selects
                 if (col < p.in) {
-                    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(p.x + (size_t)m * p.in + col));
-                    const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float2 f = __half22float2(h2[k]);
-                        xs[2 * k] = f.x; xs[2 * k + 1] = f.y;
+                    for (int u = 0; u < 4; ++u) {
+                        const __half2 pr = __ldg(reinterpret_cast<const __half2*>(p.x + (size_t)m * p.in + col + 8 * u));
+                        const float2 f = __half22float2(pr);
+                        xs[u] = f.x; xs[4 + u] = f.y;
                     }
                 } else {
 #pragma unroll

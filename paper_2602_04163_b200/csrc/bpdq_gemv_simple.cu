@@ -4,6 +4,7 @@
 // bpdq_dequant does (candidate table of Eq. 7, rounded to binary16) and accumulates
 // x * w in binary32 in column order.  No shared memory, no scratch, no tuning.
 #include "bpdq_internal.h"
+#include "bpdq_decode.cuh"
 
 #include <cuda_fp16.h>
 
@@ -23,10 +24,11 @@ gemv_simple_kernel(const uint8_t* __restrict__ blob, size_t planes_bytes, const 
     const __half* xm = x + (size_t)m * in;
     float acc = 0.f;
     for (int b = 0; b < nblocks; ++b) {
-        unsigned u[K][4];
+        unsigned u[K][4];                            // logical words of this row's units
 #pragma unroll
         for (int i = 0; i < K; ++i) {
-            const uint4 v = *reinterpret_cast<const uint4*>(blob + bpdq::plane_unit_offset(b, i, r, K, out));
+            const uint4 v = bpdq::unrotate_unit(
+                *reinterpret_cast<const uint4*>(blob + bpdq::plane_unit_offset(b, i, r, K, out)), r);
             u[i][0] = v.x; u[i][1] = v.y; u[i][2] = v.z; u[i][3] = v.w;
         }
         for (int sub = 0; sub < nsub; ++sub) {
@@ -44,26 +46,19 @@ gemv_simple_kernel(const uint8_t* __restrict__ blob, size_t planes_bytes, const 
                     if ((code >> i) & 1) a = __fadd_rn(a, c[i + 1]);
                 table[code] = __half2float(__float2half_rn(a));
             }
-            const int c_lo = (nsub == 2) ? sub * 8 : 0, c_hi = (nsub == 2) ? sub * 8 + 8 : 16;
-            for (int ch = c_lo; ch < c_hi; ++ch) {
-                const int p = (ch - r) & 15;
-                unsigned byte[K];
+            const int col_lo = (nsub == 2) ? sub * 64 : 0, col_hi = (nsub == 2) ? sub * 64 + 64 : 128;
+            for (int col = col_lo; col < col_hi; ++col) {
+                const int k = col >> 5, bit = 4 * (col & 7) + ((col >> 3) & 3);   // column = 32k + 8u + j  <->  bit 4j + u of word k
+                unsigned code = 0;
 #pragma unroll
                 for (int i = 0; i < K; ++i) {
-                    const int wsel = p >> 2;
-                    const unsigned word = wsel == 0 ? u[i][0] : wsel == 1 ? u[i][1] : wsel == 2 ? u[i][2] : u[i][3];
-                    byte[i] = (word >> (8 * (p & 3))) & 0xFFu;
+                    const unsigned word = k == 0 ? u[i][0] : k == 1 ? u[i][1] : k == 2 ? u[i][2] : u[i][3];
+                    code |= ((word >> bit) & 1u) << i;
                 }
+                float wv = table[0];
 #pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    unsigned code = 0;
-#pragma unroll
-                    for (int i = 0; i < K; ++i) code |= ((byte[i] >> t) & 1u) << i;
-                    float wv = table[0];
-#pragma unroll
-                    for (int k = 1; k < NC; ++k) wv = (code == (unsigned)k) ? table[k] : wv;
-                    acc = fmaf(__half2float(xm[b * 128 + ch * 8 + t]), wv, acc);
-                }
+                for (int kk = 1; kk < NC; ++kk) wv = (code == (unsigned)kk) ? table[kk] : wv;
+                acc = fmaf(__half2float(xm[b * 128 + col]), wv, acc);
             }
         }
     }

@@ -53,17 +53,17 @@ extern "C" int bpdq_pack(const uint8_t* bits, const uint16_t* coef, int out, int
             const uint8_t* row = bits + ((int64_t)i * out + r) * in;
             for (int64_t b = 0; b < nblocks; ++b) {
                 uint8_t* unit = dst + plane_unit_offset(b, i, r, K, out);
-                for (int c = 0; c < 16; ++c) {           // c: logical 8-column chunk of the block
-                    unsigned byte = 0;
-                    for (int t = 0; t < 8; ++t) {
-                        const unsigned v = row[b * kBlockCols + c * 8 + t];
-                        if (v > 1u)
-                            return set_error(BPDQ_ERR_INVALID, "bpdq_pack: bit value %u at plane %d row %lld col %lld",
-                                             v, i, (long long)r, (long long)(b * kBlockCols + c * 8 + t));
-                        byte |= v << t;
-                    }
-                    unit[(c - (int)(r & 15)) & 15] = (uint8_t)byte;   // byte p holds chunk (p + r) mod 16
+                uint8_t logical[16] = {0};                // logical byte L = 4*word + byte-in-word
+                for (int c = 0; c < kBlockCols; ++c) {
+                    const unsigned v = row[b * kBlockCols + c];
+                    if (v > 1u)
+                        return set_error(BPDQ_ERR_INVALID, "bpdq_pack: bit value %u at plane %d row %lld col %lld",
+                                         v, i, (long long)r, (long long)(b * kBlockCols + c));
+                    const int k = c >> 5, u = (c >> 3) & 3, j = c & 7;
+                    const int bit = 4 * j + u;            // position inside word k
+                    logical[4 * k + (bit >> 3)] |= (uint8_t)(v << (bit & 7));
                 }
+                for (int L = 0; L < 16; ++L) unit[(L - (int)(r & 15)) & 15] = logical[L];   // physical byte p holds logical byte (p + r) mod 16
             }
         }
     }
@@ -90,9 +90,11 @@ extern "C" int bpdq_unpack(const void* blob, int out, int in, int K, int group, 
             uint8_t* row = bits + ((int64_t)i * out + r) * in;
             for (int64_t b = 0; b < nblocks; ++b) {
                 const uint8_t* unit = src + plane_unit_offset(b, i, r, K, out);
-                for (int c = 0; c < 16; ++c) {
-                    const unsigned byte = unit[(c - (int)(r & 15)) & 15];
-                    for (int t = 0; t < 8; ++t) row[b * kBlockCols + c * 8 + t] = (byte >> t) & 1u;
+                for (int c = 0; c < kBlockCols; ++c) {
+                    const int k = c >> 5, u = (c >> 3) & 3, j = c & 7;
+                    const int bit = 4 * j + u;
+                    const int L = 4 * k + (bit >> 3);
+                    row[b * kBlockCols + c] = (unit[(L - (int)(r & 15)) & 15] >> (bit & 7)) & 1u;
                 }
             }
         }

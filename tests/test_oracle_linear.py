@@ -72,9 +72,10 @@ def test_unpack_reads_documented_layout():
         for i in range(K):
             for r in range(out):
                 for p in range(16):
-                    c = (p + r) % 16
-                    cols = bits[i, r, 128 * b + 8 * c: 128 * b + 8 * c + 8]
-                    planes[b, i, r, p] = sum(int(v) << t for t, v in enumerate(cols))
+                    L = (p + r) % 16
+                    k, q = divmod(L, 4)
+                    planes[b, i, r, p] = sum(int(bits[i, r, 128 * b + 32 * k + 8 * (t % 4) + 2 * q + t // 4]) << t
+                                             for t in range(8))
     cblob = np.transpose(coef, (2, 0, 1)).copy()          # [G][i][r]
     blob = np.concatenate([planes.reshape(-1), cblob.reshape(-1).view(np.uint8)])
     b2, c2 = oracle.unpack(blob, out, in_, K, g)

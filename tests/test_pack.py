@@ -31,8 +31,9 @@ def test_one_hot_bits_land_where_the_layout_says():
         blob = binding.bpdq_pack(bits, coef, g)
         nz = np.flatnonzero(blob)
         assert nz.size == 1
-        b, c, t = j // 128, (j % 128) // 8, j % 8
-        p = (c - r) % 16
+        b, k, u, jx = j // 128, (j % 128) // 32, (j % 32) // 8, j % 8
+        L, t = 4 * k + jx // 2, 4 * (jx % 2) + u          # logical byte and bit of column j
+        p = (L - r) % 16
         assert nz[0] == ((b * K + i) * out + r) * 16 + p and blob[nz[0]] == 1 << t
 
 
