@@ -1,0 +1,62 @@
+"""bpdq_gemm (TMA + tcgen05 tensor-core kernel) against the checker, same bound as every linear kernel."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2602_04163_b200 import binding, synth
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("K,g,out,in_,M", [
+    (2, 128, 128, 128, 16),      # one tile, one 128-column block, two stages
+    (2, 128, 128, 1024, 32),     # more k-blocks than pipeline stages: every barrier wraps
+    (3, 128, 256, 512, 33),      # token tile of 64 with a ragged tail
+    (1, 128, 128, 256, 5),
+    (2, 64, 128, 384, 64),       # a coefficient group per k-block
+    (3, 256, 256, 768, 100),     # a coefficient group every four k-blocks, token tile 128
+    (2, 128, 160, 640, 130),     # ragged last row tile (160 = 128 + 32), token tile 256 with a ragged tail
+    (3, 128, 384, 2048, 257),    # two token tiles of 256, the second holds one token
+    (2, 128, 1024, 1024, 300),
+    (2, 128, 128, 128, 1),       # a single token through the tensor-core path
+])
+def test_gemm_kernel(K, g, out, in_, M):
+    h, bits, coef = G.make_layer(60 + K, out, in_, K, g, max_M=M)
+    x = synth.activations(70 + K, M, in_)
+    G.check_linear(h, bits, coef, x, g, binding.KERNEL_GEMM, what="gemm")
+    y1 = G.run_linear(h, x, binding.KERNEL_GEMM)
+    y2 = G.run_linear(h, x, binding.KERNEL_GEMM)
+    assert np.array_equal(y1, y2)                        # fixed accumulation order: bit-identical reruns
+
+
+def test_gemm_equals_dequant_times_x():
+    """The decoded operand is W^ itself: with one-hot tokens the kernel must return columns of bpdq_dequant exactly."""
+    K, g, out, in_ = 3, 128, 256, 512
+    h, bits, coef = G.make_layer(5, out, in_, K, g, max_M=in_)
+    w = G.run_dequant(h).view(np.float16)
+    x = np.eye(in_, dtype=np.float16)                    # token t selects column t
+    y = G.run_linear(h, x.view(np.uint16), binding.KERNEL_GEMM)
+    assert np.array_equal(y.astype(np.float16), w.T)
+
+
+def test_dispatch_sends_large_m_to_the_tensor_core_kernel():
+    K, g, out, in_, M = 2, 128, 256, 512, 48
+    h, bits, coef = G.make_layer(9, out, in_, K, g, max_M=M)
+    x = synth.activations(10, M, in_)
+    G.check_linear(h, bits, coef, x, g, binding.KERNEL_AUTO, what="auto")
+    assert np.array_equal(G.run_linear(h, x, binding.KERNEL_AUTO), G.run_linear(h, x, binding.KERNEL_GEMM))
+
+
+@pytest.mark.parametrize("name,out,in_,K,M", [("gate", 29568, 8192, 3, 2048), ("down", 8192, 29568, 2, 512)])
+def test_gemm_full_size_sampled(name, out, in_, K, M):
+    """72B-shaped layers generated on the device; a row of every few tiles, every token, against the checker."""
+    g = 128
+    h = binding.Handle(out, in_, K, g, None, 950 + K, M)
+    x = synth.activations(951, M, in_)
+    y = G.run_linear(h, x, binding.KERNEL_GEMM)
+    rows = np.unique(np.concatenate([np.arange(0, out, 997), [0, 127, 128, out - 129, out - 128, out - 1]]))
+    y_ref, a_ref = oracle.linear(synth.plane_bits(950 + K, out, in_, K, rows),
+                                 synth.coefficients(950 + K, out, in_, K, g, rows), x, g)
+    G.assert_linear_close(y[:, rows], y_ref, a_ref, name)
+    assert np.all(np.isfinite(y))
