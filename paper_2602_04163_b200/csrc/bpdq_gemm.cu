@@ -12,15 +12,17 @@
 // 16-byte chunk c of row r is stored at chunk position c ^ (r mod 8).  TMA writes that layout by
 // itself; the decode threads reproduce it by hand.
 //
-// Roles (192 threads): warp 0 issues the TMA loads of x; warp 1 allocates TMEM and issues the
-// MMAs (one lane); warps 2..5 decode: thread = output row.  A decode thread keeps its row's plane
+// Roles (320 threads): warp 0 issues the TMA loads of x; warp 1 allocates TMEM and issues the
+// MMAs (one lane); warps 2..9 decode in two groups of four warps, thread = output row, group 0
+// taking the even 64-column stages and group 1 the odd ones (one warp per scheduler could not
+// hide its own instruction latencies).  A decode thread keeps its row's plane
 // units (K x 16 bytes per 128 columns, direct coalesced global loads, prefetched one block
 // ahead) and the 2^K candidate values of the current group (Eq. 7, the decode rule's exact
 // arithmetic) as two byte tables; eight columns cost one shift-and-mask per plane to form eight
 // code nibbles and eight byte-permutes to select and interleave the binary16 bytes, then one
-// 16-byte shared-memory store.  The same four warps run the epilogue: tcgen05.ld gives a thread
-// its output row for 16 tokens at a time; adjacent threads hold adjacent output indices, so a
-// warp writes 64 contiguous bytes of y per token.
+// 16-byte shared-memory store.  The same eight warps run the epilogue, each group on one half of
+// the token columns: tcgen05.ld gives a thread its output row for 16 tokens at a time; adjacent
+// threads hold adjacent output indices, so a warp writes 64 contiguous bytes of y per token.
 //
 // Pipeline: per stage three mbarriers -- full_b (TMA bytes landed), full_a (128 decode threads
 // arrived after a proxy fence), empty (tcgen05.commit of the MMAs that read the stage) -- and one
@@ -37,8 +39,9 @@ namespace {
 
 constexpr int BM = 128;                 // output rows per CTA (MMA M)
 constexpr int BK = 64;                  // columns per stage: one 128-byte swizzle row of binary16
-constexpr int kThreads = 192;
-constexpr int kDecodeThreads = 128;
+constexpr int kDecodeGroups = 2;
+constexpr int kDecodeThreads = 128;               // per group: one thread per output row
+constexpr int kThreads = 64 + kDecodeGroups * kDecodeThreads;
 constexpr int kATileBytes = BM * BK * 2;                       // 16 KB
 constexpr unsigned kWaitLimit = 1u << 24;                      // polls of try_wait before a wait gives up
 
@@ -217,13 +220,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
     } else {
         // ---------------- decode warps (thread = output row), then epilogue ----------------
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
+        const int grp = (warp - 2) >> 2;                 // decode group: takes the stages with kb % 2 == grp
         const int rl = quad * 32 + lane;                 // row inside the tile
         const int r = row0 + rl;
         const bool row_ok = r < p.out;
         const int rr = row_ok ? r : p.out - 1;           // clamp loads of a ragged last tile (results are not stored)
         const uint8_t* cbase = p.blob + p.planes_bytes;
         const int nblocks = p.in / 128;
-        const int kb_per_group = p.group / BK;           // 1, 2 or 4
+        const int ngroups = p.in / p.group;
+        const int gstep = p.group >= 128 ? 1 : 2;        // coefficient groups between two visits of this thread
         const size_t plane_pitch = (size_t)p.out * 16;
         const size_t coef_pitch = (size_t)p.out * 2;
 
@@ -233,66 +238,67 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
             const uint8_t* src = p.blob + (size_t)rr * 16;
 #pragma unroll
             for (int i = 0; i < K; ++i) unext[i] = __ldg(reinterpret_cast<const uint4*>(src + i * plane_pitch));
-            const uint8_t* cs = cbase + (size_t)rr * 2;
+            const int G0 = (grp * BK) / p.group;
+            const uint8_t* cs = cbase + ((size_t)G0 * (K + 1) * p.out + rr) * 2;
 #pragma unroll
             for (int i = 0; i <= K; ++i) cnext[i] = __ldg(reinterpret_cast<const unsigned short*>(cs + i * coef_pitch));
         }
         unsigned lo[2] = {0, 0}, hi[2] = {0, 0};
+        int cur_group = -1;
         const unsigned a_row = (unsigned)rl * 128u;
         const unsigned sw = (unsigned)(rl & 7);
         bool ok = true;
         for (int b = 0; b < nblocks && ok; ++b) {
-            unsigned cur[K][4];
+            unsigned cur[K][2];                          // the two logical words of this thread's half of the block
 #pragma unroll
             for (int i = 0; i < K; ++i) {
                 const uint4 u = bpdq::unrotate_unit(unext[i], rr);
-                cur[i][0] = u.x; cur[i][1] = u.y; cur[i][2] = u.z; cur[i][3] = u.w;
+                cur[i][0] = grp ? u.z : u.x;
+                cur[i][1] = grp ? u.w : u.y;
             }
             if (b + 1 < nblocks) {
                 const uint8_t* src = p.blob + ((size_t)(b + 1) * K * p.out + rr) * 16;
 #pragma unroll
                 for (int i = 0; i < K; ++i) unext[i] = __ldg(reinterpret_cast<const uint4*>(src + i * plane_pitch));
             }
+            const int kb = 2 * b + grp;
+            const int G = (kb * BK) / p.group;
+            if (G != cur_group) {                        // a new coefficient group: rebuild the candidate tables
+                cur_group = G;
+                float c[K + 1];
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const int kb = 2 * b + half;
-                if (kb % kb_per_group == 0) {            // a new coefficient group starts here
-                    float c[K + 1];
+                for (int i = 0; i <= K; ++i) c[i] = __half2float(__ushort_as_half(cnext[i]));
+                unsigned short v[1 << K];
+                bpdq::candidate_values<K>(c, v);
+                bpdq::byte_tables<K>(v, lo, hi);
+                if (G + gstep < ngroups) {
+                    const uint8_t* cs = cbase + ((size_t)(G + gstep) * (K + 1) * p.out + rr) * 2;
 #pragma unroll
-                    for (int i = 0; i <= K; ++i) c[i] = __half2float(__ushort_as_half(cnext[i]));
-                    unsigned short v[1 << K];
-                    bpdq::candidate_values<K>(c, v);
-                    bpdq::byte_tables<K>(v, lo, hi);
-                    const int G = kb / kb_per_group + 1;
-                    if (G < p.in / p.group) {
-                        const uint8_t* cs = cbase + ((size_t)G * (K + 1) * p.out + rr) * 2;
-#pragma unroll
-                        for (int i = 0; i <= K; ++i) cnext[i] = __ldg(reinterpret_cast<const unsigned short*>(cs + i * coef_pitch));
-                    }
+                    for (int i = 0; i <= K; ++i) cnext[i] = __ldg(reinterpret_cast<const unsigned short*>(cs + i * coef_pitch));
                 }
-                const int s = kb % S;
-                const unsigned ph = (unsigned)(kb / S) & 1u;
-                if (!mbar_wait(empty(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                const unsigned dst = a_base + s * kATileBytes + a_row;
-#pragma unroll
-                for (int ch = 0; ch < 8; ++ch) {         // eight 8-column chunks of this 64-column stage
-                    unsigned w[K];
-#pragma unroll
-                    for (int i = 0; i < K; ++i) w[i] = cur[i][2 * half + (ch >> 2)];
-                    const uint4 v8 = bpdq::decode8(bpdq::code_nibbles<K>(w, ch & 3), lo, hi);
-                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((unsigned)ch ^ sw) << 4)),
-                                 "r"(v8.x), "r"(v8.y), "r"(v8.z), "r"(v8.w) : "memory");
-                }
-                fence_proxy_async();                     // make the generic-proxy stores visible to the MMA's reads
-                mbar_arrive(full_a(s));
             }
+            const int s = kb % S;
+            const unsigned ph = (unsigned)(kb / S) & 1u;
+            if (!mbar_wait(empty(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+            const unsigned dst = a_base + s * kATileBytes + a_row;
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {             // eight 8-column chunks of this 64-column stage
+                unsigned w[K];
+#pragma unroll
+                for (int i = 0; i < K; ++i) w[i] = cur[i][ch >> 2];
+                const uint4 v8 = bpdq::decode8(bpdq::code_nibbles<K>(w, ch & 3), lo, hi);
+                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((unsigned)ch ^ sw) << 4)),
+                             "r"(v8.x), "r"(v8.y), "r"(v8.z), "r"(v8.w) : "memory");
+            }
+            fence_proxy_async();                         // make the generic-proxy stores visible to the MMA's reads
+            mbar_arrive(full_a(s));
         }
         // ---------------- epilogue ----------------
         if (ok && mbar_wait(acc_full, 0u, abort_flag, p.status)) {
             tc_fence_after();
             const unsigned taddr = tmem_d + ((unsigned)(quad * 32) << 16);
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 16) {
+            for (int c0 = grp * (BN / 2); c0 < (grp + 1) * (BN / 2); c0 += 16) {
                 if (tok0 + c0 >= p.M) break;             // warp-uniform
                 unsigned v[16];
                 tmem_ld16(taddr + (unsigned)c0, v);
