@@ -37,36 +37,56 @@ __device__ __forceinline__ unsigned code_nibbles(const unsigned (&w)[K], const i
     return sel;
 }
 
-// The 2^K candidate values of one (row, group) (Eq. 7) with the decode rule's arithmetic: float(c0),
-// then "+ float(ci)" in binary32 for the set bits in plane order, one rounding to binary16.
+// Codes of all 32 columns of one logical word: sel[u] holds, in nibble j, the code of column 8u + j.
 template <int K>
-__device__ __forceinline__ void candidate_values(const float (&c)[K + 1], unsigned short (&v)[1 << K]) {
+__device__ __forceinline__ void code_nibbles_word(const unsigned (&w)[K], unsigned (&sel)[4]) {
+    if constexpr (K == 2) {
+        // interleave the two planes once: e has plane 0 on even and plane 1 on odd bit positions
+        // for the columns at even positions of the word, o the same for the odd positions
+        const unsigned m = 0x55555555u;
+        const unsigned e = (w[0] & m) | ((w[1] << 1) & ~m);
+        const unsigned o = ((w[0] >> 1) & m) | (w[1] & ~m);
+        sel[0] = e & 0x33333333u;
+        sel[1] = o & 0x33333333u;
+        sel[2] = (e >> 2) & 0x33333333u;
+        sel[3] = (o >> 2) & 0x33333333u;
+    } else {
 #pragma unroll
-    for (int code = 0; code < (1 << K); ++code) {
-        float acc = c[0];
-#pragma unroll
-        for (int i = 0; i < K; ++i)
-            if ((code >> i) & 1) acc = __fadd_rn(acc, c[i + 1]);
-        v[code] = __half_as_ushort(__float2half_rn(acc));
+        for (int u = 0; u < 4; ++u) sel[u] = code_nibbles<K>(w, u);
     }
 }
 
-// Byte tables for the byte-permute decode (K <= 3): lo[0] holds the low bytes of candidates 0..3,
-// lo[1] of candidates 4..7 (zero when K < 3); hi[] the high bytes.
+// The 2^K candidate values of one (row, group) (Eq. 7) with the decode rule's arithmetic: float(c0),
+// then "+ float(ci)" in binary32 for the set bits in plane order, one rounding to binary16.
+// Returned as byte tables for the byte-permute decode (K <= 3): lo[0] holds the low bytes of
+// candidates 0..3, lo[1] of candidates 4..7 (zero when K < 3); hi[] the high bytes.
 template <int K>
-__device__ __forceinline__ void byte_tables(const unsigned short (&v)[1 << K], unsigned (&lo)[2], unsigned (&hi)[2]) {
+__device__ __forceinline__ void candidate_byte_tables(const float (&c)[K + 1], unsigned (&lo)[2], unsigned (&hi)[2]) {
     static_assert(K >= 1 && K <= 3, "byte-permute decode covers at most eight candidates");
-    lo[0] = lo[1] = hi[0] = hi[1] = 0u;
+    float acc[1 << K];
 #pragma unroll
-    for (int e = 0; e < (1 << K); ++e) {
-        lo[e >> 2] |= (unsigned)(v[e] & 0xFFu) << (8 * (e & 3));
-        hi[e >> 2] |= (unsigned)(v[e] >> 8) << (8 * (e & 3));
+    for (int code = 0; code < (1 << K); ++code) {
+        float a = c[0];
+#pragma unroll
+        for (int i = 0; i < K; ++i)
+            if ((code >> i) & 1) a = __fadd_rn(a, c[i + 1]);
+        acc[code] = a;
     }
+    unsigned pair[4] = {0u, 0u, 0u, 0u};             // candidates (2q, 2q+1) as two binary16 in one register
+#pragma unroll
+    for (int q = 0; q < (1 << K) / 2 || q < 1; ++q) {
+        const __half2 h = __floats2half2_rn(acc[2 * q], (2 * q + 1) < (1 << K) ? acc[2 * q + 1] : 0.f);
+        pair[q] = *reinterpret_cast<const unsigned*>(&h);
+    }
+    lo[0] = __byte_perm(pair[0], pair[1], 0x6420u);
+    hi[0] = __byte_perm(pair[0], pair[1], 0x7531u);
+    lo[1] = __byte_perm(pair[2], pair[3], 0x6420u);
+    hi[1] = __byte_perm(pair[2], pair[3], 0x7531u);
 }
 
 // Eight binary16 values (columns in order) from eight code nibbles.
 __device__ __forceinline__ uint4 decode8(const unsigned sel, const unsigned (&lo)[2], const unsigned (&hi)[2]) {
-    const unsigned sel_hi = sel >> 16;
+    const unsigned sel_hi = __umulhi(sel, 0x10000u);         // sel >> 16 on the multiplier instead of the shifter
     const unsigned l0 = __byte_perm(lo[0], lo[1], sel), h0 = __byte_perm(hi[0], hi[1], sel);
     const unsigned l1 = __byte_perm(lo[0], lo[1], sel_hi), h1 = __byte_perm(hi[0], hi[1], sel_hi);
     uint4 o;

@@ -14,18 +14,23 @@
 //
 // Roles (320 threads): warp 0 issues the TMA loads of x; warp 1 allocates TMEM and issues the
 // MMAs (one lane); warps 2..9 decode in two groups of four warps, thread = output row, group 0
-// taking the even 64-column stages and group 1 the odd ones (one warp per scheduler could not
-// hide its own instruction latencies).  A decode thread keeps its row's plane
-// units (K x 16 bytes per 128 columns, direct coalesced global loads, prefetched one block
-// ahead) and the 2^K candidate values of the current group (Eq. 7, the decode rule's exact
-// arithmetic) as two byte tables; eight columns cost one shift-and-mask per plane to form eight
+// taking the even 128-column blocks (two stages each) and group 1 the odd ones (one warp per
+// scheduler could not hide its own instruction latencies).  The packed planes and coefficients of a stage come
+// through the same pipeline as x: for every stage the producer also issues bulk copies of the K
+// plane segments (128 rows x 16 bytes, contiguous in the blob; once per 128-column block, with
+// the block's first stage) and the K+1 coefficient segments (128 rows x 2 bytes) of the tile's rows, so that no decode thread ever waits on global memory.
+// A decode thread reads its row's units and coefficients from the stage, builds the 2^K
+// candidate values of the group (Eq. 7, the decode rule's exact arithmetic) as two byte tables,
+// and then eight columns cost one shift-and-mask per plane to form eight
 // code nibbles and eight byte-permutes to select and interleave the binary16 bytes, then one
 // 16-byte shared-memory store.  The same eight warps run the epilogue, each group on one half of
 // the token columns: tcgen05.ld gives a thread its output row for 16 tokens at a time; adjacent
 // threads hold adjacent output indices, so a warp writes 64 contiguous bytes of y per token.
 //
-// Pipeline: per stage three mbarriers -- full_b (TMA bytes landed), full_a (128 decode threads
-// arrived after a proxy fence), empty (tcgen05.commit of the MMAs that read the stage) -- and one
+// Pipeline: per stage four mbarriers -- full_b (x tile landed), full_p (planes and coefficients
+// landed; the producer issued them after `empty`, so the stage's A slot is free as well), full_a
+// (128 decode threads arrived after a proxy fence), empty (tcgen05.commit of the MMAs that read
+// the stage) -- and one
 // acc_full barrier for the epilogue.  Every wait is bounded: on expiry the thread records
 // BPDQ_ERR_TIMEOUT in the handle's status word, raises a CTA-wide abort flag that lets all other
 // waits fall through, and the CTA still runs to its common exit where TMEM is freed.
@@ -45,12 +50,15 @@ constexpr int kThreads = 64 + kDecodeGroups * kDecodeThreads;
 constexpr int kATileBytes = BM * BK * 2;                       // 16 KB
 constexpr unsigned kWaitLimit = 1u << 24;                      // polls of try_wait before a wait gives up
 
-template <int BN> struct Cfg {
+template <int K, int BN> struct Cfg {
     static constexpr int kBTileBytes = BN * BK * 2;
-    static constexpr int kStageBytes = kATileBytes + kBTileBytes;
-    static constexpr int kStages = (200 * 1024) / kStageBytes > 8 ? 8 : (200 * 1024) / kStageBytes;
+    static constexpr int kPlaneBytes = K * BM * 16;             // K segments of 128 rows x 16 bytes
+    static constexpr int kCoefBytes = (K + 1) * BM * 2;         // K+1 segments of 128 rows x 2 bytes
+    static constexpr int kPackedBytes = (kPlaneBytes + kCoefBytes + 1023) / 1024 * 1024;
+    static constexpr int kStageBytes = kATileBytes + kBTileBytes + kPackedBytes;
+    static constexpr int kStages = (222 * 1024) / kStageBytes > 8 ? 8 : (222 * 1024) / kStageBytes;
     static constexpr int kTmemCols = BN < 32 ? 32 : BN;        // power of two >= 32
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
 };
 
 struct GemmParams {
@@ -102,6 +110,10 @@ __device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
+__device__ __forceinline__ void bulk_load(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(unsigned dst_smem, unsigned cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
 }
@@ -147,19 +159,21 @@ __host__ __device__ constexpr unsigned instr_desc_f16(int m, int n) {
 template <int K, int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
-    using C = Cfg<BN>;
+    using C = Cfg<K, BN>;
     constexpr int S = C::kStages;
     extern __shared__ unsigned char smem_raw[];
     const unsigned base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* smem = smem_raw + (base - smem_u32(smem_raw));
     const unsigned a_base = base;                                  // S x 16 KB
     const unsigned b_base = base + S * kATileBytes;                // S x BN*128 bytes
-    const unsigned bar_base = b_base + S * C::kBTileBytes;
+    const unsigned p_base = b_base + S * C::kBTileBytes;           // S x (planes, coefficients)
+    const unsigned bar_base = p_base + S * C::kPackedBytes;
     auto full_b = [&](int s) { return bar_base + 8u * s; };
     auto full_a = [&](int s) { return bar_base + 8u * (S + s); };
     auto empty = [&](int s) { return bar_base + 8u * (2 * S + s); };
-    const unsigned acc_full = bar_base + 8u * (3 * S);
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(smem + (bar_base - base) + 8 * (3 * S + 1));
+    auto full_p = [&](int s) { return bar_base + 8u * (3 * S + s); };
+    const unsigned acc_full = bar_base + 8u * (4 * S);
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(smem + (bar_base - base) + 8 * (4 * S + 1));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -172,6 +186,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
             mbar_init(full_b(s), 1);
             mbar_init(full_a(s), kDecodeThreads);
             mbar_init(empty(s), 1);
+            mbar_init(full_p(s), 1);
         }
         mbar_init(acc_full, 1);
         *abort_flag = 0;
@@ -187,12 +202,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
     const unsigned tmem_d = *tmem_slot;
 
     if (warp == 0) {
-        // ---------------- TMA producer: x tiles ----------------
+        // ---------------- producer: x tiles (TMA), plane and coefficient segments (bulk copies) ----------------
         if (lane == 0) {
+            const int nrows = min(BM, p.out - row0);     // ragged last row tile: a multiple of 16
+            const unsigned seg_p = (unsigned)nrows * 16u, seg_c = (unsigned)nrows * 2u;
+            const uint8_t* cbase = p.blob + p.planes_bytes;
             for (int kb = 0; kb < nkb; ++kb) {
                 const int s = kb % S;
                 const unsigned ph = (unsigned)(kb / S) & 1u;
                 if (!mbar_wait(empty(s), ph ^ 1u, abort_flag, p.status)) break;
+                // packed operands first: the decode threads are the longer leg of the pipeline
+                const bool first_half = (kb & 1) == 0;   // the block's plane units travel with its first stage
+                mbar_expect_tx(full_p(s), (first_half ? (unsigned)K * seg_p : 0u) + (unsigned)(K + 1) * seg_c);
+                const unsigned pdst = p_base + s * C::kPackedBytes;
+                const int b = kb >> 1, G = (kb * BK) / p.group;
+                if (first_half) {
+#pragma unroll
+                    for (int i = 0; i < K; ++i)
+                        bulk_load(pdst + i * (BM * 16), p.blob + (((size_t)b * K + i) * p.out + row0) * 16, seg_p, full_p(s));
+                }
+#pragma unroll
+                for (int i = 0; i <= K; ++i)
+                    bulk_load(pdst + C::kPlaneBytes + i * (BM * 2), cbase + (((size_t)G * (K + 1) + i) * p.out + row0) * 2, seg_c, full_p(s));
                 mbar_expect_tx(full_b(s), C::kBTileBytes);
                 tma_load_2d(b_base + s * C::kBTileBytes, &x_map, kb * BK, tok0, full_b(s));
             }
@@ -223,75 +254,59 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
         const int grp = (warp - 2) >> 2;                 // decode group: takes the stages with kb % 2 == grp
         const int rl = quad * 32 + lane;                 // row inside the tile
         const int r = row0 + rl;
-        const bool row_ok = r < p.out;
-        const int rr = row_ok ? r : p.out - 1;           // clamp loads of a ragged last tile (results are not stored)
-        const uint8_t* cbase = p.blob + p.planes_bytes;
+        const bool row_ok = r < p.out;                   // rows past a ragged last tile decode stale bytes; nothing of theirs is stored
         const int nblocks = p.in / 128;
-        const int ngroups = p.in / p.group;
-        const int gstep = p.group >= 128 ? 1 : 2;        // coefficient groups between two visits of this thread
-        const size_t plane_pitch = (size_t)p.out * 16;
-        const size_t coef_pitch = (size_t)p.out * 2;
-
-        uint4 unext[K];
-        unsigned short cnext[K + 1];
-        {
-            const uint8_t* src = p.blob + (size_t)rr * 16;
+        unsigned a_off[8];                               // swizzled byte offset of each 16-byte chunk of this thread's row
 #pragma unroll
-            for (int i = 0; i < K; ++i) unext[i] = __ldg(reinterpret_cast<const uint4*>(src + i * plane_pitch));
-            const int G0 = (grp * BK) / p.group;
-            const uint8_t* cs = cbase + ((size_t)G0 * (K + 1) * p.out + rr) * 2;
-#pragma unroll
-            for (int i = 0; i <= K; ++i) cnext[i] = __ldg(reinterpret_cast<const unsigned short*>(cs + i * coef_pitch));
-        }
-        unsigned lo[2] = {0, 0}, hi[2] = {0, 0};
-        int cur_group = -1;
-        const unsigned a_row = (unsigned)rl * 128u;
-        const unsigned sw = (unsigned)(rl & 7);
+        for (int ch = 0; ch < 8; ++ch) a_off[ch] = (unsigned)rl * 128u + (((unsigned)ch ^ (unsigned)(rl & 7)) << 4);
         bool ok = true;
-        for (int b = 0; b < nblocks && ok; ++b) {
-            unsigned cur[K][2];                          // the two logical words of this thread's half of the block
+        for (int b = grp; b < nblocks && ok; b += kDecodeGroups) {
+            unsigned cur[K][4];                          // logical words of this row's plane units
+            unsigned lo[2], hi[2];
 #pragma unroll
-            for (int i = 0; i < K; ++i) {
-                const uint4 u = bpdq::unrotate_unit(unext[i], rr);
-                cur[i][0] = grp ? u.z : u.x;
-                cur[i][1] = grp ? u.w : u.y;
-            }
-            if (b + 1 < nblocks) {
-                const uint8_t* src = p.blob + ((size_t)(b + 1) * K * p.out + rr) * 16;
+            for (int half = 0; half < 2; ++half) {
+                const int kb = 2 * b + half;
+                const int s = kb % S;
+                const unsigned ph = (unsigned)(kb / S) & 1u;
+                if (!mbar_wait(full_p(s), ph, abort_flag, p.status)) { ok = false; break; }
+                const unsigned psrc = p_base + s * C::kPackedBytes;
+                if (half == 0) {
 #pragma unroll
-                for (int i = 0; i < K; ++i) unext[i] = __ldg(reinterpret_cast<const uint4*>(src + i * plane_pitch));
-            }
-            const int kb = 2 * b + grp;
-            const int G = (kb * BK) / p.group;
-            if (G != cur_group) {                        // a new coefficient group: rebuild the candidate tables
-                cur_group = G;
-                float c[K + 1];
-#pragma unroll
-                for (int i = 0; i <= K; ++i) c[i] = __half2float(__ushort_as_half(cnext[i]));
-                unsigned short v[1 << K];
-                bpdq::candidate_values<K>(c, v);
-                bpdq::byte_tables<K>(v, lo, hi);
-                if (G + gstep < ngroups) {
-                    const uint8_t* cs = cbase + ((size_t)(G + gstep) * (K + 1) * p.out + rr) * 2;
-#pragma unroll
-                    for (int i = 0; i <= K; ++i) cnext[i] = __ldg(reinterpret_cast<const unsigned short*>(cs + i * coef_pitch));
+                    for (int i = 0; i < K; ++i) {
+                        uint4 raw;
+                        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(raw.x), "=r"(raw.y), "=r"(raw.z), "=r"(raw.w)
+                                     : "r"(psrc + i * (BM * 16) + rl * 16));
+                        const uint4 u = bpdq::unrotate_unit(raw, r);
+                        cur[i][0] = u.x; cur[i][1] = u.y; cur[i][2] = u.z; cur[i][3] = u.w;
+                    }
                 }
-            }
-            const int s = kb % S;
-            const unsigned ph = (unsigned)(kb / S) & 1u;
-            if (!mbar_wait(empty(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-            const unsigned dst = a_base + s * kATileBytes + a_row;
+                if (half == 0 || p.group == 64) {        // candidate tables of the coefficient group that starts here
+                    float c[K + 1];
 #pragma unroll
-            for (int ch = 0; ch < 8; ++ch) {             // eight 8-column chunks of this 64-column stage
-                unsigned w[K];
+                    for (int i = 0; i <= K; ++i) {
+                        unsigned short hbits;
+                        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(hbits) : "r"(psrc + C::kPlaneBytes + i * (BM * 2) + rl * 2));
+                        c[i] = __half2float(__ushort_as_half(hbits));
+                    }
+                    bpdq::candidate_byte_tables<K>(c, lo, hi);
+                }
+                const unsigned dst = a_base + s * kATileBytes;
 #pragma unroll
-                for (int i = 0; i < K; ++i) w[i] = cur[i][ch >> 2];
-                const uint4 v8 = bpdq::decode8(bpdq::code_nibbles<K>(w, ch & 3), lo, hi);
-                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((unsigned)ch ^ sw) << 4)),
-                             "r"(v8.x), "r"(v8.y), "r"(v8.z), "r"(v8.w) : "memory");
+                for (int wd = 0; wd < 2; ++wd) {         // two 32-column words per 64-column stage
+                    unsigned w[K], sel[4];
+#pragma unroll
+                    for (int i = 0; i < K; ++i) w[i] = cur[i][2 * half + wd];
+                    bpdq::code_nibbles_word<K>(w, sel);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const uint4 v8 = bpdq::decode8(sel[u], lo, hi);
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + a_off[4 * wd + u]),
+                                     "r"(v8.x), "r"(v8.y), "r"(v8.z), "r"(v8.w) : "memory");
+                    }
+                }
+                fence_proxy_async();                     // make the generic-proxy stores visible to the MMA's reads
+                mbar_arrive(full_a(s));
             }
-            fence_proxy_async();                         // make the generic-proxy stores visible to the MMA's reads
-            mbar_arrive(full_a(s));
         }
         // ---------------- epilogue ----------------
         if (ok && mbar_wait(acc_full, 0u, abort_flag, p.status)) {
@@ -344,7 +359,7 @@ EncodeTiledFn encode_tiled_fn() {
 
 template <int K, int BN>
 int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
-    using C = Cfg<BN>;
+    using C = Cfg<K, BN>;
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemm_kernel<K, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
