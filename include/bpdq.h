@@ -87,6 +87,7 @@ enum {
 };
 
 #define BPDQ_GEMV_MAX_M 16
+#define BPDQ_NOALLOC_MAX_OUT 65536   /* most output rows bpdq_linear_noalloc accepts */
 
 /* Storage accounting (paper: Table 1, column BPW = K + 16 (K+1) / g bits per weight).
  * Bytes of the packed blob: out*in*K/8 + out*(in/g)*(K+1)*2.  Returns 0 for an unsupported
@@ -133,6 +134,29 @@ BPDQ_API int bpdq_linear_ex(bpdq_handle_t h, const void* x_fp16_dev, void* y_fp1
  * the stream.  Pinned host memory makes the copies asynchronous up to that wait. */
 BPDQ_API int bpdq_linear_host(bpdq_handle_t h, const void* x_fp16_host, void* y_fp16_host, int M,
                      void* stream);
+
+/* The look-up-table kernel without a handle and without any allocation.  (The paper has no
+ * counterpart: this entry point exists for callers that cannot allocate device memory at the
+ * time they need the layer -- a plug-in whose host application reserves all device memory up
+ * front and hands out one arena that already holds the packed weights, a process running under
+ * a memory budget in which a later cudaMalloc may fail, or a latency-critical loop in which the
+ * implicit device synchronisation of an allocation is not acceptable.)
+ *
+ * blob_dev is the packed blob (layout above, bpdq_packed_bytes() bytes) already in DEVICE memory,
+ * caller-owned; x [M][in] and y [M][out] as for bpdq_linear, 0 <= M <= BPDQ_GEMV_MAX_M.  All
+ * three pointers 16-byte aligned.  The kernel's scratch (binary32 row sums, arrival counters,
+ * status word) is a static device array inside the library, about 0.5 MB, held by every GPU
+ * that loads the library until the process exits; it bounds the layer at
+ * out <= BPDQ_NOALLOC_MAX_OUT rows (larger: BPDQ_ERR_INVALID, nothing is launched).  Shapes as
+ * for bpdq_create, with group 128 or 256.
+ *
+ * The first call on a device looks up the array's device address and two device attributes;
+ * make that first call outside any stream capture.  No call allocates or frees device or host
+ * memory.  Every call on a device uses the same array: it is cleared on `stream` before the
+ * kernel runs, so two calls that overlap on the GPU (different streams, different threads)
+ * race on it -- issue them on one stream.  Asynchronous like bpdq_linear. */
+BPDQ_API int bpdq_linear_noalloc(const void* blob_dev, int out, int in, int K, int group, const void* x_fp16_dev,
+                        void* y_fp16_dev, int M, void* stream);
 
 /* Sets the largest M that bpdq_linear sends to the look-up-table kernel (0 = always use the
  * tensor-core kernel; at most BPDQ_GEMV_MAX_M). */

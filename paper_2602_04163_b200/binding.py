@@ -18,10 +18,11 @@ LIB_PATH = os.path.join(_PKG, "libbpdq.so")
 OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(6)
 KERNEL_AUTO, KERNEL_GEMV, KERNEL_GEMM, KERNEL_GEMV_SIMPLE = range(4)
 GEMV_MAX_M = 16
+NOALLOC_MAX_OUT = 65536
 
 EXPORTS = ("bpdq_packed_bytes", "bpdq_pack", "bpdq_unpack", "bpdq_create", "bpdq_dequant", "bpdq_linear",
            "bpdq_linear_ex", "bpdq_linear_host", "bpdq_set_gemv_max_m", "bpdq_read_blob", "bpdq_get_status",
-           "bpdq_launch_count", "bpdq_destroy", "bpdq_last_error")
+           "bpdq_launch_count", "bpdq_destroy", "bpdq_last_error", "bpdq_linear_noalloc")
 
 _lib = None
 
@@ -50,6 +51,7 @@ def lib() -> ctypes.CDLL:
         L.bpdq_linear.argtypes = [vp, vp, vp, i, vp]
         L.bpdq_linear_ex.argtypes = [vp, vp, vp, i, i, vp]
         L.bpdq_linear_host.argtypes = [vp, vp, vp, i, vp]
+        L.bpdq_linear_noalloc.argtypes = [vp, i, i, i, i, vp, vp, i, vp]
         L.bpdq_set_gemv_max_m.argtypes = [vp, i]
         L.bpdq_read_blob.argtypes = [vp, vp]
         L.bpdq_get_status.argtypes = [vp, vp]
@@ -104,6 +106,12 @@ def bpdq_unpack(blob: np.ndarray, out: int, in_: int, K: int, group: int):
     coef = np.empty((K + 1, out, in_ // group), dtype=np.uint16)
     _check(lib().bpdq_unpack(_np_ptr(blob), out, in_, K, group, _np_ptr(bits), _np_ptr(coef)))
     return bits, coef
+
+
+def bpdq_linear_noalloc(blob_ptr: int, out: int, in_: int, K: int, group: int, x_ptr: int, y_ptr: int, M: int,
+                        stream: int = 0) -> None:
+    """Look-up-table kernel on a caller-owned device blob; uses the library's static scratch, allocates nothing."""
+    _check(lib().bpdq_linear_noalloc(blob_ptr, out, in_, K, group, x_ptr, y_ptr, M, stream))
 
 
 class Handle:

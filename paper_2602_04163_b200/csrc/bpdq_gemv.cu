@@ -449,3 +449,90 @@ int launch_gemv(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t st
 }
 
 }  // namespace bpdq
+
+// ---------------------------------------------------------------------------------------------
+// bpdq_linear_noalloc: the look-up-table kernel for callers that must not allocate.
+// ---------------------------------------------------------------------------------------------
+// The kernel's scratch (binary32 row sums, arrival counters, status word) lives in a file-scope
+// device array instead of a handle.  In host code `g_noalloc_scratch` is only a stand-in for the
+// symbol: its device address is fetched with cudaGetSymbolAddress, once per device, and that
+// address is what the kernel receives.
+namespace {
+
+constexpr size_t kNoallocWsBytes = (size_t)kMaxMT * BPDQ_NOALLOC_MAX_OUT * sizeof(float);
+constexpr size_t kNoallocCounterBytes = ((size_t)BPDQ_NOALLOC_MAX_OUT / 16 / kChunkRgs) * sizeof(unsigned);
+constexpr size_t kNoallocBytes = kNoallocWsBytes + kNoallocCounterBytes + 256;   // + status word
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoallocBytes];
+
+constexpr int kMaxDevices = 64;
+struct NoallocDevice {
+    bool ready;
+    unsigned char* scratch;       // device address of g_noalloc_scratch on this device
+    int sm_count, smem_optin;
+};
+NoallocDevice g_noalloc_dev[kMaxDevices];
+
+// Set-up of the current device: symbol address and the two device attributes the launcher needs.
+int noalloc_setup(int dev) {
+    NoallocDevice& d = g_noalloc_dev[dev];
+    if (d.ready) return BPDQ_OK;
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+    if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "bpdq_linear_noalloc: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+    int major = 0;
+    if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess ||
+        (e = cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess ||
+        (e = cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
+        return bpdq::set_error(BPDQ_ERR_CUDA, "bpdq_linear_noalloc: device attributes: %s", cudaGetErrorString(e));
+    if (major != 10)
+        return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear_noalloc: device is sm_%dx, this library is built for sm_100a only", major);
+    d.scratch = static_cast<unsigned char*>(ptr);
+    d.ready = true;
+    return BPDQ_OK;
+}
+
+}  // namespace
+
+extern "C" int bpdq_linear_noalloc(const void* blob_dev, int out, int in, int K, int group, const void* x_fp16_dev,
+                                   void* y_fp16_dev, int M, void* stream) {
+    using namespace bpdq;
+    if (M < 0 || M > BPDQ_GEMV_MAX_M)
+        return set_error(BPDQ_ERR_INVALID, "bpdq_linear_noalloc: M=%d outside [0, %d]", M, BPDQ_GEMV_MAX_M);
+    if (!shape_supported(out, in, K, group) || !gemv_supported(out, in, K, group))
+        return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear_noalloc: unsupported shape out=%d in=%d K=%d g=%d", out, in, K, group);
+    if (out > BPDQ_NOALLOC_MAX_OUT)
+        return set_error(BPDQ_ERR_INVALID, "bpdq_linear_noalloc: out=%d exceeds the static scratch limit of %d rows", out,
+                         BPDQ_NOALLOC_MAX_OUT);
+    if (M == 0) return BPDQ_OK;
+    if (!blob_dev || !x_fp16_dev || !y_fp16_dev) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_noalloc: null pointer");
+    if ((reinterpret_cast<uintptr_t>(blob_dev) | reinterpret_cast<uintptr_t>(x_fp16_dev) | reinterpret_cast<uintptr_t>(y_fp16_dev)) & 15u)
+        return set_error(BPDQ_ERR_INVALID, "bpdq_linear_noalloc: blob, x and y must be 16-byte aligned");
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear_noalloc: no CUDA device (%s)", cudaGetErrorString(e));
+    if (dev < 0 || dev >= kMaxDevices) return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear_noalloc: device ordinal %d", dev);
+    int rc = noalloc_setup(dev);
+    if (rc != BPDQ_OK) return rc;
+    const NoallocDevice& d = g_noalloc_dev[dev];
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    // The scratch keeps whatever the last call left; the kernel needs row sums and counters at zero.
+    const size_t ws_used = (size_t)kMaxMT * out * sizeof(float);
+    if ((e = cudaMemsetAsync(d.scratch, 0, ws_used, s)) != cudaSuccess ||
+        (e = cudaMemsetAsync(d.scratch + kNoallocWsBytes, 0, kNoallocCounterBytes + 256, s)) != cudaSuccess)
+        return set_error(BPDQ_ERR_CUDA, "bpdq_linear_noalloc: clearing the scratch: %s", cudaGetErrorString(e));
+
+    bpdq_handle_s h{};                                   // a view for the launcher; owns nothing
+    h.out = out; h.in = in; h.K = K; h.group = group; h.max_M = BPDQ_GEMV_MAX_M; h.device = dev;
+    h.sm_count = d.sm_count; h.smem_optin = d.smem_optin;
+    h.d_blob = const_cast<uint8_t*>(static_cast<const uint8_t*>(blob_dev));
+    h.planes_bytes = planes_bytes(out, in, K);
+    h.blob_bytes = h.planes_bytes + coefs_bytes(out, in, K, group);
+    h.d_ws = reinterpret_cast<float*>(d.scratch);
+    h.ws_bytes = ws_used;
+    h.d_counters = reinterpret_cast<unsigned*>(d.scratch + kNoallocWsBytes);
+    h.n_counters = gemv_counter_count(out);
+    h.d_status = reinterpret_cast<int*>(d.scratch + kNoallocWsBytes + kNoallocCounterBytes);
+    return launch_gemv(&h, x_fp16_dev, y_fp16_dev, M, s);
+}
