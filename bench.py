@@ -286,6 +286,7 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
 
     if rank == 0 and not args.no_extras:
         line["sections"] = extra_sections(torch, binding, args, peaks, sp, stream)
+        line["sections"]["decode_sweep_80_layers_K2"] = full_stack_section(torch, binding, peaks, sp, stream)
     for L in layers:
         L.destroy()
 
@@ -352,7 +353,105 @@ def extra_sections(torch, binding, args, peaks, sp, stream):
                                      "frac_measured": b / (med * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         h.bpdq_destroy()
         del w
+
+    def xt(M, in_, seed=3):
+        return torch.from_numpy(synth.activations(seed, M, in_).view(np.int16).copy()).cuda().view(torch.float16)
+
+    # decoder layer with fused handles (q|k|v share x, gate|up share x): 4 launches instead of 7, same bytes
+    for K in (2, 3):
+        fused = [("qkv", 10240, 8192), ("o", 8192, 8192), ("gate_up", 59136, 8192), ("down", 8192, 29568)]
+        copies = 3
+        layers = [[binding.Handle(o, i, K, GROUP, None, 500 + 10 * c + li, 1) for li, (_, o, i) in enumerate(fused)] for c in range(copies)]
+        xs = {8192: xt(1, 8192), 29568: xt(1, 29568)}
+        ys = {o: torch.empty((1, o), dtype=torch.float16, device="cuda") for _, o, _ in fused}
+        b = sum(useful_bytes(o, i, K, GROUP, 1) for _, o, i in fused)
+        n = 60
+
+        def run_layers():
+            for k in range(n):
+                for h in layers[k % copies]:
+                    h.bpdq_linear(xs[h.in_].data_ptr(), ys[h.out].data_ptr(), 1, sp)
+        run_layers()
+        ms = event_time_ms(torch, run_layers, stream) / n
+        out[f"gemv_layer_fused_handles_K{K}"] = {"launches_per_layer": 4, "us_per_layer": ms * 1e3, "gbs": b / (ms * 1e-3) / 1e9,
+                                                 "frac_measured": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                                 "l2": f"{copies} layer copies of {b / 1e6:.0f} MB rotated"}
+        for L in layers:
+            for h in L:
+                h.bpdq_destroy()
+
+    # token-count sweep on the gate and down projections: both kernels, to place the dispatch threshold
+    sweep = []
+    for K in (2, 3):
+        for name, o, i in (("gate", 29568, 8192), ("down", 8192, 29568)):
+            h = binding.Handle(o, i, K, GROUP, None, 13, 64)
+            for M in (1, 2, 4, 8, 16, 32, 64):
+                x = xt(M, i)
+                y = torch.empty((M, o), dtype=torch.float16, device="cuda")
+                rec = {"linear": name, "K": K, "M": M}
+                for kname, kid in (("lut", binding.KERNEL_GEMV), ("tensor", binding.KERNEL_GEMM)):
+                    if kid == binding.KERNEL_GEMV and M > binding.GEMV_MAX_M:
+                        continue
+                    med, _ = timed(lambda: h.bpdq_linear_ex(x.data_ptr(), y.data_ptr(), M, kid, sp), 5)
+                    rec[f"us_{kname}"] = med * 1e3
+                best = min(v for k, v in rec.items() if k.startswith("us_"))
+                rec["gbs_best"] = useful_bytes(o, i, K, GROUP, M) / (best * 1e-6) / 1e9
+                sweep.append(rec)
+            h.bpdq_destroy()
+    out["token_sweep"] = sweep
+
+    # prefill on the tensor-core kernel: one 72B-shaped layer at K = 3, M = 2048 and M = 8192
+    shapes = synth.QWEN25_72B_LAYER
+    for K, M in ((3, 2048), (3, 8192), (2, 8192)):
+        hs = [binding.Handle(o, i, K, GROUP, None, 700 + li, M) for li, (_, o, i) in enumerate(shapes)]
+        xs = {8192: xt(M, 8192), 29568: xt(M, 29568)}
+        ys = {o: torch.empty((M, o), dtype=torch.float16, device="cuda") for o in sorted({o for _, o, _ in shapes})}
+        flops = sum(2.0 * M * o * i for _, o, i in shapes)
+
+        def run_prefill():
+            for h in hs:
+                h.bpdq_linear(xs[h.in_].data_ptr(), ys[h.out].data_ptr(), M, sp)
+        run_prefill()
+        ts = sorted(event_time_ms(torch, run_prefill, stream) for _ in range(3))
+        ms = ts[1]
+        per = []
+        for (name, o, i), h in zip(shapes, hs):
+            if name in ("gate", "down", "q"):
+                t1 = sorted(event_time_ms(torch, lambda: h.bpdq_linear(xs[i].data_ptr(), ys[o].data_ptr(), M, sp), stream) for _ in range(3))[1]
+                per.append({"linear": name, "ms": t1, "tflops": 2.0 * M * o * i / (t1 * 1e-3) / 1e12})
+        tf = flops / (ms * 1e-3) / 1e12
+        out[f"prefill_gemm_layer_K{K}_M{M}"] = {
+            "ms_per_layer": ms, "tflops": tf, "per_linear": per,
+            "roofline": {"bound": "tensor", "kernel": "gemm_kernel", "achieved": tf, "peak": peaks["tflops"], "unit": "TFLOP/s",
+                         "frac": tf / peaks["tflops"], "frac_of_sustained": tf / peaks["tflops_sustained"],
+                         "peak_source": peaks["source"] + " bf16 burst (fp16 has the same nominal rate)", "traffic": None}}
+        for h in hs:
+            h.bpdq_destroy()
+        del xs, ys
     return out
+
+
+def full_stack_section(torch, binding, peaks, sp, stream, n_layers=80):
+    """All linears of an 80-layer 72B-shaped stack (K = 2, about 20.8 GB packed), one token through each."""
+    shapes, K = synth.QWEN25_72B_LAYER, 2
+    hs = []
+    for layer in range(n_layers):
+        for li, (_, o, i) in enumerate(shapes):
+            hs.append(binding.Handle(o, i, K, GROUP, None, synth.linear_seed(5, layer, li, K), 1))
+    xs = {i: torch.from_numpy(synth.activations(9, 1, i).view(np.int16).copy()).cuda().view(torch.float16) for i in (8192, 29568)}
+    ys = {o: torch.empty((1, o), dtype=torch.float16, device="cuda") for o in sorted({o for _, o, _ in shapes})}
+
+    def sweep():
+        for h in hs:
+            h.bpdq_linear(xs[h.in_].data_ptr(), ys[h.out].data_ptr(), 1, sp)
+    sweep()
+    ms = sorted(event_time_ms(torch, sweep, stream) for _ in range(3))[1]
+    b = n_layers * layer_bytes(shapes, K, 1)
+    res = {"layers": n_layers, "linears": len(hs), "packed_gb": sum(h.packed_bytes for h in hs) / 1e9, "ms_per_sweep": ms,
+           "gbs": b / (ms * 1e-3) / 1e9, "frac_measured": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    for h in hs:
+        h.bpdq_destroy()
+    return res
 
 
 def main():

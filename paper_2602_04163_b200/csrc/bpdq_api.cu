@@ -64,7 +64,7 @@ extern "C" int bpdq_create(bpdq_handle_t* hp, int out, int in, int K, int group,
     h->blob_bytes = h->planes_bytes + coefs_bytes(out, in, K, group);
     h->ws_bytes = gemv_workspace_bytes(out, in, K, group, max_M, h->sm_count);
     h->n_counters = gemv_counter_count(out);
-    h->gemv_max_m = 2;
+    h->gemv_max_m = 6;   // measured crossover on 72B-shaped layers: three two-token passes of the look-up-table kernel still beat the tensor-core kernel
 
     const size_t stage_x = (size_t)max_M * in * 2, stage_y = (size_t)max_M * out * 2;
     if ((e = cudaMalloc(&h->d_blob, h->blob_bytes)) != cudaSuccess ||

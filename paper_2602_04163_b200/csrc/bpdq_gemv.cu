@@ -6,20 +6,23 @@
 //     y[r] = sum_G ( c0[r,G] * X_G  +  sum_i ci[r,G] * S_i[r,G] ),
 //     X_G = sum of x over group G,    S_i[r,G] = sum of x_j over the set bits of plane i in G.
 //
-// S_i is read from look-up tables instead of being added bit by bit: for every 8 consecutive
-// inputs ("chunk") the 256 subset sums of x are precomputed in shared memory (binary32), so one
-// plane BYTE costs one byte-permute (address), one shared-memory load and one add.
+// S_i is read from look-up tables instead of being added bit by bit: for every 8 inputs that share
+// a plane byte ("chunk") the 256 subset sums of x are precomputed in shared memory (binary32), so
+// one plane BYTE costs one byte-permute (address), one shared-memory load and half a packed add.
 //
 // Work split.  A CTA owns a slice of 512 input columns (4 blocks of 128) and a range of 16-row
 // groups; it builds the 64 chunk tables of its slice once (64 KB per token) and then streams
-// planes.  A warp takes 16 rows x 4 blocks: lane (h, a) = (lane/16, lane%16) owns row a and the
-// two blocks of parity h; its 16-byte plane units and coefficients arrive through a per-warp
-// cp.async ring several tasks deep (HBM latency is covered by bytes in flight, not by registers),
-// and it walks the 16 bytes of each unit.  The blob stores, at byte p of row r, the 8-column chunk ("logical byte") (p + r) mod 16,
-// and table entries are laid out as [entry][slot], slot = 16*block + chunk, so at every step the
-// 32 lanes of a warp hit 32 different banks whatever the data: table loads are conflict-free by
-// construction.  The tables start at a multiple of 64 KB in the shared window, so the byte-permute
-// that splices the plane byte into bits 8..15 of the lane's slot address yields the final address.
+// planes.  A warp takes 16 rows x 4 blocks per task: lane (h, a) = (lane/16, lane%16) owns row a
+// and the two blocks of parity h.  Its 16-byte plane units and binary16 coefficients come straight
+// from global memory into registers (16 lanes x 16 bytes = 256 contiguous bytes per request), two
+// or three tasks ahead, so that HBM latency is covered by loads in flight and shared memory
+// carries nothing but the look-ups.  The blob stores, at byte p of row r, the 8-column chunk
+// ("logical byte") (p + r) mod 16, and table entries are laid out as [entry][slot],
+// slot = 16*block + chunk, so at every step the 32 lanes of a warp hit 32 different banks whatever
+// the data: table loads are conflict-free by construction.  The tables start at a multiple of
+// 64 KB in the shared window, so the byte-permute that splices the plane byte into bits 8..15 of
+// the lane's slot address yields the final address.  Look-up results are accumulated two at a
+// time with packed binary32 adds.
 // Row sums are combined across slices with binary32 atomic adds into a small workspace
 // [token][row] that lives in L2; per 128 rows an arrival counter tells the CTA that delivers the
 // last contribution to round those rows to binary16, write y and zero the workspace again.
@@ -35,7 +38,6 @@ constexpr int kSlots = 16 * kSliceBlocks;             // chunk tables per slice 
 constexpr int kTableBytes = 256 * kSlots * 4;         // one token's tables: 64 KB
 constexpr int kMaxMT = 2;                             // tokens per pass (64 KB of tables each)
 constexpr int kChunkRgs = 8;                          // row groups (of 16 rows) per completion counter
-constexpr int kMaxStages = 8;                         // depth limit of a warp's staging ring
 constexpr int kMiscBytes = 4096;                      // xsum + completion list, at the start of shared memory
 constexpr int kMaxDone = 512;                         // completed chunks handled per batch
 
@@ -53,51 +55,34 @@ struct GemvParams {
     int dyn_smem;                // dynamic shared memory bytes of the launch
 };
 
-// One stage of a warp's staging ring holds one task (16 rows x 4 blocks): the lanes' plane units
-// ([q][plane][lane] x 16 bytes, each lane copies its own) and the task's coefficients
-// ([block][coefficient][row] binary16: 4(K+1) runs of 32 bytes, copied as 16-byte halves by the
-// first 8(K+1) lanes).  Coefficients are read by other lanes than copied them, so the warp
-// synchronises after its cp.async groups have landed.
+// Registers of one task (16 rows x 4 blocks) of a lane: K plane units and K+1 coefficients for
+// each of its two blocks.
 template <int K>
-struct Stage {
-    static constexpr int kPlaneBytes = 2 * K * 32 * 16;
-    static constexpr int kCoefSegs = kSliceBlocks * (K + 1);          // 32-byte runs per task
-    static constexpr int kCoefBytes = (kCoefSegs * 32 + 127) / 128 * 128;
-    static constexpr int kBytes = kPlaneBytes + kCoefBytes;
+struct Task {
+    uint4 pl[2][K];
+    unsigned short cf[2][K + 1];
 };
 
-__device__ __forceinline__ void cp_async16(unsigned dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async4(unsigned dst, const void* src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_dyn(int pending) {
-    switch (pending) {
-        case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
-        case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
-        case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
-        case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
-        case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
-        case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
-        case 6: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
-        default: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
-    }
-}
-__device__ __forceinline__ uint4 lds_v4(unsigned addr) {
+__device__ __forceinline__ uint4 ldg_stream16(const uint8_t* p) {
     uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
-__device__ __forceinline__ unsigned short lds_u16(unsigned addr) {
+// volatile, so that it stays ahead of the weight requests issued after it
+__device__ __forceinline__ unsigned ldg_first4(const void* p) {
+    unsigned v;
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ unsigned short ldg_stream2(const uint8_t* p) {
     unsigned short v;
-    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+    asm volatile("ld.global.nc.L1::no_allocate.u16 %0, [%1];" : "=h"(v) : "l"(p));
     return v;
 }
 // Table load.  Not volatile: its address is computed from plane bytes that were read after the
 // barrier that published the tables, so it cannot move above that barrier, and the compiler may
-// interleave the 32 independent look-ups of a plane unit freely.
+// interleave the independent look-ups of a plane unit freely.
 template <int IMM>
 __device__ __forceinline__ float lds_table(unsigned addr) {
     float v;
@@ -107,41 +92,38 @@ __device__ __forceinline__ float lds_table(unsigned addr) {
 __device__ __forceinline__ unsigned word_of(const uint4& v, int k) {
     return k == 0 ? v.x : k == 1 ? v.y : k == 2 ? v.z : v.w;
 }
+// A pair of binary32 accumulators in one 64-bit register: (lo, hi) += (a, b) as one packed add.
+__device__ __forceinline__ void add2(unsigned long long& acc, float a, float b) {
+    asm("{\n\t.reg .b64 t;\n\tmov.b64 t, {%1, %2};\n\tadd.rn.f32x2 %0, %0, t;\n\t}" : "+l"(acc) : "f"(a), "f"(b));
+}
+__device__ __forceinline__ float2 unpack2(unsigned long long v) {
+    float2 f;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(f.x), "=f"(f.y) : "l"(v));
+    return f;
+}
 
-template <int K, int MT, int W>
+template <int K, int MT, int D, int W>
 __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p) {
     constexpr int kThreads = W * 32;
+    constexpr int NS = K * MT;                        // look-up streams per step: (plane, token) pairs
+    constexpr int NP = (NS + 1) / 2;                  // packed accumulators
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int h = lane >> 4, a = lane & 15;
 
     // ---- shared memory map (addresses in the shared window) ----
     //   [smem0, +kMiscBytes)             xsum, completion list
-    //   [.., lut0)                       staging slots (low region)
-    //   [lut0, lut0 + MT*64 KB)          tables, lut0 a multiple of 64 KB
-    //   [.., smem0 + dyn_smem)           staging slots (high region)
+    //   [lut0, lut0 + MT*64 KB)          tables, lut0 the next multiple of 64 KB
     const unsigned smem0 = (unsigned)__cvta_generic_to_shared(smem);
     const unsigned lut0 = (smem0 + kMiscBytes + 65535u) & ~65535u;
-    const unsigned low0 = smem0 + kMiscBytes;
-    const int nlow = (int)(lut0 - low0) / Stage<K>::kBytes;
-    const unsigned high0 = lut0 + MT * kTableBytes;
-    const int nhigh = ((int)(smem0 + p.dyn_smem) - (int)high0) / Stage<K>::kBytes;
-    int stages = (nlow + (nhigh > 0 ? nhigh : 0)) / W;
-    if (stages > kMaxStages) stages = kMaxStages;
-    if ((int)(smem0 + p.dyn_smem) < (int)high0 || stages < 1) {   // tables or one slot per warp do not fit
+    if (lut0 + MT * kTableBytes > smem0 + (unsigned)p.dyn_smem) {       // tables do not fit
         if (tid == 0) atomicExch(p.status, BPDQ_ERR_UNSUPPORTED);
-        return;                                                    // uniform: no barrier has been reached
+        return;                                                          // uniform: no barrier has been reached
     }
     float* xsum = reinterpret_cast<float*>(smem);                         // [MT][kSliceBlocks]
     int* done = reinterpret_cast<int*>(smem + 64);                        // [kMaxDone]
     int* ndone = done + kMaxDone;
     float* lut = reinterpret_cast<float*>(smem + (lut0 - smem0));         // [MT][256][kSlots]
-
-    // slot address of stage j of this warp
-    auto slot_addr = [&](int j) -> unsigned {
-        const int k = wid * stages + j;
-        return k < nlow ? low0 + k * Stage<K>::kBytes : high0 + (k - nlow) * Stage<K>::kBytes;
-    };
 
     // the lane's table-slot address per step: lut0 + 4*((s + a) mod 16) + 64*h; the plane byte is
     // spliced into bits 8..15 (entry row stride 256 B)
@@ -155,6 +137,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
     const int t_end = t + p.tasks_base + (bid < p.tasks_rem ? 1 : 0);
     const uint8_t* cbase = p.blob + p.planes_bytes;
     const size_t plane_pitch = (size_t)p.out * 16;    // bytes between planes of one block
+    const size_t coef_pitch = (size_t)p.out * 2;      // bytes between coefficients of one group
 
     while (t < t_end) {
         const int s = t / p.nrg;
@@ -164,79 +147,68 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
 
         // per-lane source pointers of the first task; a task further on is W*16 rows further on
         const uint8_t* psrc[2];
+        const uint8_t* csrc[2];
         bool valid[2];
         {
             const int r = (rg_begin + wid) * 16 + a;
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 const int b = s * kSliceBlocks + 2 * q + h;
-                valid[q] = b < p.nblocks;
-                psrc[q] = p.blob + ((size_t)b * K * p.out + r) * 16;
+                valid[q] = b < p.nblocks;                                  // false past the end of a ragged last slice
+                const int bb = valid[q] ? b : 0;
+                psrc[q] = p.blob + ((size_t)bb * K * p.out + r) * 16;
+                const int G = (bb * 128) / p.group;
+                csrc[q] = cbase + ((size_t)G * (K + 1) * p.out + r) * 2;
             }
         }
-        // coefficient runs: copy slot L (one per lane, two rounds when 8(K+1) > 32) is half (L & 1)
-        // of run L >> 1 = (block, coefficient)
-        constexpr int kCoefRounds = (Stage<K>::kCoefSegs * 2 + 31) / 32;
-        const uint8_t* csrc[kCoefRounds];
-        int cstate[kCoefRounds];                      // 0: no copy, 1: copy, 2: zero-fill
-#pragma unroll
-        for (int c = 0; c < kCoefRounds; ++c) {
-            const int L = c * 32 + lane, seg = L >> 1;
-            const int blk = seg / (K + 1), i = seg - blk * (K + 1);
-            const int b = s * kSliceBlocks + blk;
-            const int G = (b * 128) / p.group;
-            cstate[c] = (seg >= Stage<K>::kCoefSegs) ? 0 : (b < p.nblocks ? 1 : 2);
-            csrc[c] = cbase + (((size_t)G * (K + 1) + i) * p.out + (size_t)(rg_begin + wid) * 16) * 2 + (L & 1) * 16;
-        }
-        auto issue_task = [&](int n, unsigned dst) {
+        auto load_task = [&](Task<K>& tk, int n) {
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
-                const unsigned pdst = dst + (q * K) * 512 + lane * 16;
                 if (valid[q]) {
                     const uint8_t* ps = psrc[q] + (size_t)n * (W * 256);
 #pragma unroll
-                    for (int i = 0; i < K; ++i) cp_async16(pdst + i * 512, ps + i * plane_pitch);
-                } else {                              // block past the end of a ragged last slice
+                    for (int i = 0; i < K; ++i) tk.pl[q][i] = ldg_stream16(ps + i * plane_pitch);
+                    const uint8_t* cs = csrc[q] + (size_t)n * (W * 32);
 #pragma unroll
-                    for (int i = 0; i < K; ++i)
-                        asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(pdst + i * 512), "r"(0u) : "memory");
+                    for (int i = 0; i <= K; ++i) tk.cf[q][i] = ldg_stream2(cs + i * coef_pitch);
+                } else {                              // contributes nothing: zero planes, zero coefficients
+#pragma unroll
+                    for (int i = 0; i < K; ++i) tk.pl[q][i] = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                    for (int i = 0; i <= K; ++i) tk.cf[q][i] = 0;
                 }
-            }
-#pragma unroll
-            for (int c = 0; c < kCoefRounds; ++c) {
-                const unsigned cdst = dst + Stage<K>::kPlaneBytes + (c * 32 + lane) * 16;
-                if (cstate[c] == 1) cp_async16(cdst, csrc[c] + (size_t)n * (W * 32));
-                else if (cstate[c] == 2)
-                    asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(cdst), "r"(0u) : "memory");
             }
         };
 
-        // the first tasks are requested before the tables are built, to overlap the latency
-        for (int n = 0; n < stages - 1; ++n) {
-            if (n < ntask) issue_task(n, slot_addr(n));
-            cp_async_commit();
-        }
+        // ---- this thread's inputs for the table build come first, then the first tasks' weights: the
+        // weight requests of 148 CTAs would otherwise queue ahead of the few bytes of x ----
+        static_assert(kSlots * 8 == W * 32, "one table item (slot, entry block) per thread");
+        const int slot = tid & (kSlots - 1);          // chunk table
+        const int eh = tid >> 6;                      // entries eh*32 .. eh*32+31 share inputs 5..7
+        // slot = 16*block + logical byte L; L = 4k + q is byte q of 32-column word k, and bit
+        // 4*jj + u of that byte is column 32k + 8u + 2q + jj: four pairs of adjacent inputs
+        const int col = s * (kSliceBlocks * 128) + (slot >> 2) * 32 + (slot & 3) * 2;
+        unsigned xraw[MT][4];
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                xraw[m][u] = col < p.in ? ldg_first4(p.x + (size_t)m * p.in + col + 8 * u) : 0u;
+
+        Task<K> tk[D];
+#pragma unroll
+        for (int d = 0; d < D; ++d)
+            if (d < ntask) load_task(tk[d], d);
 
         // ---- build the 64 chunk tables of this slice (per token) ----
-        for (int item = tid; item < kSlots * 8; item += kThreads) {
-            const int slot = item & (kSlots - 1);     // chunk table
-            const int eh = item >> 6;                 // entries eh*32 .. eh*32+31 share inputs 5..7
-            // slot = 16*block + logical byte L; L = 4k + q is byte q of 32-column word k, and bit
-            // 4*jj + u of that byte is column 32k + 8u + 2q + jj: four pairs of adjacent inputs
-            const int col = s * (kSliceBlocks * 128) + (slot >> 2) * 32 + (slot & 3) * 2;
+        {
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
                 float xs[8];                          // xs[t]: the input that bit t of the plane byte selects
-                if (col < p.in) {
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const __half2 pr = __ldg(reinterpret_cast<const __half2*>(p.x + (size_t)m * p.in + col + 8 * u));
-                        const float2 f = __half22float2(pr);
-                        xs[u] = f.x; xs[4 + u] = f.y;
-                    }
-                } else {
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) xs[k] = 0.f;
+                for (int u = 0; u < 4; ++u) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&xraw[m][u]));
+                    xs[u] = f.x; xs[4 + u] = f.y;
                 }
                 float lo[32];                         // subset sums of inputs 0..4
                 lo[0] = 0.f;
@@ -263,60 +235,62 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
         __syncthreads();
 
         // ---- stream the row groups of this slice ----
-        int stage_rd = 0, stage_wr = stages - 1;
-        for (int n = 0; n < ntask; ++n) {
-            {
-                const int nn = n + stages - 1;
-                if (nn < ntask) issue_task(nn, slot_addr(stage_wr));
-                cp_async_commit();
-                stage_wr = (stage_wr + 1 == stages) ? 0 : stage_wr + 1;
-            }
-            cp_async_wait_dyn(stages - 1);            // all but the newest stages-1 groups are complete: task n has landed
-            __syncwarp();                             // ... for every lane: coefficients are read across lanes
-            const unsigned st_base = slot_addr(stage_rd);
-            stage_rd = (stage_rd + 1 == stages) ? 0 : stage_rd + 1;
-
+        auto process_task = [&](const Task<K>& tk, int n) {
             float yacc[MT];
 #pragma unroll
             for (int m = 0; m < MT; ++m) yacc[m] = 0.f;
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
-                float S[K][MT][2];                    // two partial sums per plane shorten the add chains
-                uint4 pl[K];
+                // stream sidx = i*MT + m; streams are added in pairs, and every pair keeps two
+                // accumulators (even and odd steps) to shorten the add chains
+                unsigned long long acc[NP][2];
 #pragma unroll
-                for (int i = 0; i < K; ++i) {
-                    pl[i] = lds_v4(st_base + (q * K + i) * 512 + lane * 16);
-#pragma unroll
-                    for (int m = 0; m < MT; ++m) S[i][m][0] = S[i][m][1] = 0.f;
-                }
+                for (int j = 0; j < NP; ++j) acc[j][0] = acc[j][1] = 0ull;
+                float held = 0.f;                     // odd stream count: the last stream pairs two steps
 #pragma unroll
                 for (int st = 0; st < 16; ++st) {
+                    float v[NS];
 #pragma unroll
                     for (int i = 0; i < K; ++i) {
                         // address = slot address with the plane byte in bits 8..15
-                        const unsigned addr = __byte_perm(word_of(pl[i], st >> 2), off[st], 0x7604u | ((st & 3) << 4));
+                        const unsigned addr = __byte_perm(word_of(tk.pl[q][i], st >> 2), off[st], 0x7604u | ((st & 3) << 4));
 #pragma unroll
                         for (int m = 0; m < MT; ++m) {      // the token's table and the block pair go into the immediate
-                            if (m == 0 && q == 0) S[i][m][st & 1] += lds_table<0>(addr);
-                            else if (m == 0) S[i][m][st & 1] += lds_table<128>(addr);
-                            else if (q == 0) S[i][m][st & 1] += lds_table<kTableBytes>(addr);
-                            else S[i][m][st & 1] += lds_table<kTableBytes + 128>(addr);
+                            if (m == 0 && q == 0) v[i * MT + m] = lds_table<0>(addr);
+                            else if (m == 0) v[i * MT + m] = lds_table<128>(addr);
+                            else if (q == 0) v[i * MT + m] = lds_table<kTableBytes>(addr);
+                            else v[i * MT + m] = lds_table<kTableBytes + 128>(addr);
                         }
                     }
+#pragma unroll
+                    for (int j = 0; j < NS / 2; ++j) add2(acc[j][st & 1], v[2 * j], v[2 * j + 1]);
+                    if (NS & 1) {
+                        if ((st & 1) == 0) held = v[NS - 1];
+                        else add2(acc[NP - 1][(st >> 1) & 1], held, v[NS - 1]);
+                    }
+                }
+                float S[NS];
+#pragma unroll
+                for (int j = 0; j < NS / 2; ++j) {
+                    const float2 e = unpack2(acc[j][0]), o = unpack2(acc[j][1]);
+                    S[2 * j] = e.x + o.x;
+                    S[2 * j + 1] = e.y + o.y;
+                }
+                if (NS & 1) {
+                    const float2 e = unpack2(acc[NP - 1][0]), o = unpack2(acc[NP - 1][1]);
+                    S[NS - 1] = (e.x + e.y) + (o.x + o.y);
                 }
                 const int blk = 2 * q + h;
-                const unsigned cw = st_base + Stage<K>::kPlaneBytes + (blk * (K + 1)) * 32 + a * 2;
-                const float c0 = __half2float(__ushort_as_half(lds_u16(cw)));
+                const float c0 = __half2float(__ushort_as_half(tk.cf[q][0]));
 #pragma unroll
                 for (int m = 0; m < MT; ++m) yacc[m] = fmaf(c0, xsum[m * kSliceBlocks + blk], yacc[m]);
 #pragma unroll
                 for (int i = 0; i < K; ++i) {
-                    const float ci = __half2float(__ushort_as_half(lds_u16(cw + (i + 1) * 32)));
+                    const float ci = __half2float(__ushort_as_half(tk.cf[q][i + 1]));
 #pragma unroll
-                    for (int m = 0; m < MT; ++m) yacc[m] = fmaf(ci, S[i][m][0] + S[i][m][1], yacc[m]);
+                    for (int m = 0; m < MT; ++m) yacc[m] = fmaf(ci, S[i * MT + m], yacc[m]);
                 }
             }
-            __syncwarp();                             // the stage is refilled by the next iteration's copies
             // the two half-warps hold the even-block and odd-block parts of the same 16 rows
 #pragma unroll
             for (int m = 0; m < MT; ++m) yacc[m] += __shfl_xor_sync(0xffffffffu, yacc[m], 16);
@@ -325,8 +299,17 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
 #pragma unroll
                 for (int m = 0; m < MT; ++m) atomicAdd(&p.ws[(size_t)m * p.out + r], yacc[m]);
             }
+        };
+        for (int n0 = 0; n0 < ntask; n0 += D) {
+#pragma unroll
+            for (int d = 0; d < D; ++d) {
+                const int n = n0 + d;
+                if (n < ntask) {                      // warp-uniform
+                    process_task(tk[d], n);
+                    if (n + D < ntask) load_task(tk[d], n + D);
+                }
+            }
         }
-        cp_async_wait_dyn(0);
 
         // ---- hand this segment over ----
         // Row sums are accumulated across slices with binary32 atomic adds in `ws` (kept zero
@@ -369,12 +352,14 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
     }
 }
 
-template <int K, int MT, int W>
+template <int K, int MT, int D, int W>
 int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     static int configured_smem = 0;
-    const int smem = h->smem_optin;
+    const int smem = 65536 + MT * kTableBytes;        // tables start at the first 64 KB boundary of the shared window
+    if (smem > h->smem_optin)
+        return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv: %d bytes of shared memory needed, device offers %d", smem, h->smem_optin);
     if (configured_smem != smem) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<K, MT, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<K, MT, D, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemv: shared memory opt-in: %s", cudaGetErrorString(e));
         configured_smem = smem;
     }
@@ -385,20 +370,17 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     p.tasks_base = (int)(total / grid);
     p.tasks_rem = (int)(total % grid);
     p.dyn_smem = smem;
-    gemv_lut_kernel<K, MT, W><<<grid, W * 32, smem, stream>>>(p);
+    gemv_lut_kernel<K, MT, D, W><<<grid, W * 32, smem, stream>>>(p);
     h->launches += 1;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemv launch: %s", cudaGetErrorString(e));
     return BPDQ_OK;
 }
 
-// Warps per CTA: 16 when at least two ring stages per warp fit beside the tables, else 8.
+// Tasks kept in flight per lane: three while their registers fit (K <= 2), else two.
 template <int K, int MT>
 int launch_one(bpdq_handle_s* h, const GemvParams& p, cudaStream_t stream) {
-    const int ring_bytes = h->smem_optin - 2048 - kMiscBytes - MT * kTableBytes;   // 2 KB: allowance for the window base
-    if (ring_bytes / (16 * Stage<K>::kBytes) >= 2) return launch_cfg<K, MT, 16>(h, p, stream);
-    if (ring_bytes / (8 * Stage<K>::kBytes) >= 1) return launch_cfg<K, MT, 8>(h, p, stream);
-    return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv: staging ring does not fit (K=%d, tokens=%d)", K, MT);
+    return launch_cfg<K, MT, (K <= 2 ? 3 : 2), 16>(h, p, stream);
 }
 
 template <int K>
