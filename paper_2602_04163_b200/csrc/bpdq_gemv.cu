@@ -53,6 +53,7 @@ struct GemvParams {
     int nblocks, nslices, nrg;
     int tasks_base, tasks_rem;   // task range of CTA b: b*base + min(b, rem), one longer for b < rem
     int dyn_smem;                // dynamic shared memory bytes of the launch
+    int early_weights;           // the packed weights were complete before the preceding kernel of the stream started
 };
 
 // Registers of one task (16 rows x 4 blocks) of a lane: K plane units and K+1 coefficients for
@@ -110,6 +111,12 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int h = lane >> 4, a = lane & 15;
+
+    // Programmatic dependent launch: the next kernel of the stream may be scheduled as soon as this
+    // one's CTAs leave their SMs; everything this kernel itself reads or writes that an earlier
+    // kernel may have produced (x, y, the workspace) is touched only after griddepcontrol.wait below.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    bool dep_waited = false;
 
     // ---- shared memory map (addresses in the shared window) ----
     //   [smem0, +kMiscBytes)             xsum, completion list
@@ -180,25 +187,37 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
             }
         };
 
-        // ---- this thread's inputs for the table build come first, then the first tasks' weights: the
-        // weight requests of 148 CTAs would otherwise queue ahead of the few bytes of x ----
+        // ---- this thread's inputs for the table build and the first tasks' weights ----
         static_assert(kSlots * 8 == W * 32, "one table item (slot, entry block) per thread");
         const int slot = tid & (kSlots - 1);          // chunk table
         const int eh = tid >> 6;                      // entries eh*32 .. eh*32+31 share inputs 5..7
         // slot = 16*block + logical byte L; L = 4k + q is byte q of 32-column word k, and bit
         // 4*jj + u of that byte is column 32k + 8u + 2q + jj: four pairs of adjacent inputs
         const int col = s * (kSliceBlocks * 128) + (slot >> 2) * 32 + (slot & 3) * 2;
+        // Before the first wait on the preceding kernel only the weights may be requested (they
+        // belong to the handle and were complete long ago); then x, which that kernel may have written.
+        Task<K> tk[D];
+        const bool early = !dep_waited && p.early_weights != 0;
+        if (early) {
+#pragma unroll
+            for (int d = 0; d < D; ++d)
+                if (d < ntask) load_task(tk[d], d);
+        }
+        if (!dep_waited) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            dep_waited = true;
+        }
         unsigned xraw[MT][4];
 #pragma unroll
         for (int m = 0; m < MT; ++m)
 #pragma unroll
             for (int u = 0; u < 4; ++u)
                 xraw[m][u] = col < p.in ? ldg_first4(p.x + (size_t)m * p.in + col + 8 * u) : 0u;
-
-        Task<K> tk[D];
+        if (!early) {
 #pragma unroll
-        for (int d = 0; d < D; ++d)
-            if (d < ntask) load_task(tk[d], d);
+            for (int d = 0; d < D; ++d)
+                if (d < ntask) load_task(tk[d], d);
+        }
 
         // ---- build the 64 chunk tables of this slice (per token) ----
         {
@@ -370,9 +389,15 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     p.tasks_base = (int)(total / grid);
     p.tasks_rem = (int)(total % grid);
     p.dyn_smem = smem;
-    gemv_lut_kernel<K, MT, D, W><<<grid, W * 32, smem, stream>>>(p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(W * 32); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // lets this launch overlap the tail of the kernel before it
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_lut_kernel<K, MT, D, W>, p);
     h->launches += 1;
-    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemv launch: %s", cudaGetErrorString(e));
     return BPDQ_OK;
 }
@@ -415,6 +440,7 @@ int launch_gemv(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t st
     p.ws = h->d_ws;
     p.counters = h->d_counters;
     p.status = h->d_status;
+    p.early_weights = h->caller_blob ? 0 : 1;
     p.out = h->out; p.in = h->in; p.group = h->group;
     p.nblocks = h->in / 128;
     p.nslices = (p.nblocks + kSliceBlocks - 1) / kSliceBlocks;
@@ -509,6 +535,7 @@ extern "C" int bpdq_linear_noalloc(const void* blob_dev, int out, int in, int K,
     h.out = out; h.in = in; h.K = K; h.group = group; h.max_M = BPDQ_GEMV_MAX_M; h.device = dev;
     h.sm_count = d.sm_count; h.smem_optin = d.smem_optin;
     h.d_blob = const_cast<uint8_t*>(static_cast<const uint8_t*>(blob_dev));
+    h.caller_blob = 1;                                  // the caller may have produced it with the kernel just before this one
     h.planes_bytes = planes_bytes(out, in, K);
     h.blob_bytes = h.planes_bytes + coefs_bytes(out, in, K, group);
     h.d_ws = reinterpret_cast<float*>(d.scratch);

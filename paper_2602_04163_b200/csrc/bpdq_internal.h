@@ -40,6 +40,7 @@ struct bpdq_handle_s {
     int sm_count;
     int smem_optin;           // largest dynamic shared memory a CTA may opt in to
     uint8_t* d_blob;          // planes then coefficients
+    int caller_blob;          // 1: d_blob belongs to the caller (bpdq_linear_noalloc), its contents may be recent
     size_t blob_bytes, planes_bytes;
     float* d_ws;              // binary32 row sums of the split over input slices (zero between calls)
     size_t ws_bytes;
