@@ -207,10 +207,17 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
     xs = {in_: torch.from_numpy(synth.activations(7, 1, in_).view(np.int16).copy()).cuda().view(torch.float16)
           for in_ in sorted({i for _, _, i in shapes})}
     ys = {out: torch.empty((1, out), dtype=torch.float16, device="cuda") for out in sorted({o for _, o, _ in shapes})}
+    ys_each = [torch.empty((1, o), dtype=torch.float16, device="cuda") for _, o, _ in shapes]
+    x_ptrs = [xs[i].data_ptr() for _, _, i in shapes]
+    y_ptrs = [y.data_ptr() for y in ys_each]
 
     def step(layer):
-        for (name, h) in layer.handles:
-            h.bpdq_linear(xs[h.in_].data_ptr(), ys[h.out].data_ptr(), M, sp)
+        # the layer's seven linears have independent inputs in this workload: one launch covers them all
+        binding.bpdq_linear_batch([h for _, h in layer.handles], x_ptrs, y_ptrs, M, sp)
+
+    def step_separate(layer):
+        for k, (name, h) in enumerate(layer.handles):
+            h.bpdq_linear(x_ptrs[k], y_ptrs[k], M, sp)
 
     launches0 = sum(h.bpdq_launch_count() for L in layers for _, h in L.handles)
     for w in range(args.warmup):
@@ -273,7 +280,8 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": "qwen2.5-72b-shaped decoder layer, K=2, g=128, M=1 (7 linears: q k v o gate up down)",
+            "config": {"workload": "qwen2.5-72b-shaped decoder layer, K=2, g=128, M=1 (7 linears: q k v o gate up down, each with its own x, "
+                                   "issued as one bpdq_linear_batch call; sections.seven_separate_calls times seven bpdq_linear calls)",
                        "l2": f"inputs larger than L2: {copies} distinct layer copies of {bytes_step / 1e6:.1f} MB rotated between steps",
                        "useful_bytes_per_step": bytes_step, "parallelism": "replicas only" if world > 1 else "single GPU"},
             "e2e": {"value": e2e_value, "unit": UNIT,
@@ -282,10 +290,25 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
             "roofline": {"bound": "hbm", "kernel": "gemv_lut_kernel", "achieved": per_gpu, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": per_gpu / peaks["hbm_gbs"], "peak_source": peaks["source"],
                          "frac_of_nominal_8tbs": per_gpu / HBM_NOMINAL_GBS, "traffic": None,
-                         "launches_per_step": len(shapes), "algorithmic_bytes_per_launch_avg": bytes_step / len(shapes)}}
+                         "launches_per_step": 1, "algorithmic_bytes_per_launch": bytes_step}}
+
+    # the same layer as seven separate bpdq_linear calls
+    for w in range(3):
+        step_separate(layers[w % copies])
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for s_ in range(args.steps):
+        step_separate(layers[s_ % copies])
+    e1.record(stream)
+    e1.synchronize()
+    ms_sep = e0.elapsed_time(e1) / args.steps
+    separate = {"launches_per_layer": len(shapes), "us_per_layer": ms_sep * 1e3, "gbs": bytes_step / (ms_sep * 1e-3) / 1e9,
+                "frac_measured": bytes_step / (ms_sep * 1e-3) / 1e9 / peaks["hbm_gbs"]}
 
     if rank == 0 and not args.no_extras:
         line["sections"] = extra_sections(torch, binding, args, peaks, sp, stream)
+        line["sections"]["seven_separate_calls"] = separate
         line["sections"]["decode_sweep_80_layers_K2"] = full_stack_section(torch, binding, peaks, sp, stream)
     for L in layers:
         L.destroy()
@@ -376,6 +399,32 @@ def extra_sections(torch, binding, args, peaks, sp, stream):
         out[f"gemv_layer_fused_handles_K{K}"] = {"launches_per_layer": 4, "us_per_layer": ms * 1e3, "gbs": b / (ms * 1e-3) / 1e9,
                                                  "frac_measured": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                                  "l2": f"{copies} layer copies of {b / 1e6:.0f} MB rotated"}
+        for L in layers:
+            for h in L:
+                h.bpdq_destroy()
+
+    # the same layer through bpdq_linear_batch: one launch for all seven linears (legitimate when, as in this
+    # benchmark, every linear has its own input), and the grouping a decoder allows: {q,k,v} {o} {gate,up} {down}
+    for K in (2, 3):
+        shapes7 = synth.QWEN25_72B_LAYER
+        copies = 3
+        layers = [[binding.Handle(o, i, K, GROUP, None, 800 + 10 * c + li, 1) for li, (_, o, i) in enumerate(shapes7)] for c in range(copies)]
+        xs = {8192: xt(1, 8192), 29568: xt(1, 29568)}
+        ys = [torch.empty((1, o), dtype=torch.float16, device="cuda") for _, o, _ in shapes7]
+        b = layer_bytes(shapes7, K, 1)
+        n = 60
+        for label, groups in (("one_launch", [[0, 1, 2, 3, 4, 5, 6]]), ("decoder_groups", [[0, 1, 2], [3], [4, 5], [6]])):
+            def run_batched():
+                for k in range(n):
+                    hs = layers[k % copies]
+                    for grp in groups:
+                        binding.bpdq_linear_batch([hs[j] for j in grp], [xs[hs[j].in_].data_ptr() for j in grp],
+                                                  [ys[j].data_ptr() for j in grp], 1, sp)
+            run_batched()
+            ms = event_time_ms(torch, run_batched, stream) / n
+            out[f"gemv_layer_batched_{label}_K{K}"] = {"launches_per_layer": len(groups), "us_per_layer": ms * 1e3,
+                                                       "gbs": b / (ms * 1e-3) / 1e9, "frac_measured": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                                       "l2": f"{copies} layer copies of {b / 1e6:.0f} MB rotated"}
         for L in layers:
             for h in L:
                 h.bpdq_destroy()

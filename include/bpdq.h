@@ -87,6 +87,7 @@ enum {
 };
 
 #define BPDQ_GEMV_MAX_M 16
+#define BPDQ_BATCH_MAX 16            /* most linears bpdq_linear_batch takes in one call */
 #define BPDQ_NOALLOC_MAX_OUT 65536   /* most output rows bpdq_linear_noalloc accepts */
 
 /* Storage accounting (paper: Table 1, column BPW = K + 16 (K+1) / g bits per weight).
@@ -128,6 +129,19 @@ BPDQ_API int bpdq_linear(bpdq_handle_t h, const void* x_fp16_dev, void* y_fp16_d
  * M > BPDQ_GEMV_MAX_M is BPDQ_ERR_INVALID. */
 BPDQ_API int bpdq_linear_ex(bpdq_handle_t h, const void* x_fp16_dev, void* y_fp16_dev, int M, int kernel,
                    void* stream);
+
+/* Several independent linears in one launch of the look-up-table kernel (decode: q, k, v of one
+ * token, or gate and up, or a whole layer's linears when their inputs do not depend on each
+ * other).  y[k] = x[k] * W^[k]^T for k = 0..n-1, each exactly as bpdq_linear with
+ * BPDQ_KERNEL_GEMV computes it; the task spaces of the n linears are concatenated, so launch
+ * ramp, table set-up and tail are paid once instead of n times.  hs, xs, ys are HOST arrays of n
+ * handles / device pointers (read before the call returns); 1 <= n <= BPDQ_BATCH_MAX; the
+ * handles are distinct, live on the current device, share K and have group 128 or 256;
+ * 0 <= M <= min(max_M of every handle, BPDQ_GEMV_MAX_M).  Inputs may be shared between
+ * linears; outputs must not overlap anything else.  BPDQ_ERR_INVALID / BPDQ_ERR_UNSUPPORTED
+ * otherwise, with nothing launched. */
+BPDQ_API int bpdq_linear_batch(const bpdq_handle_t* hs, const void* const* xs_fp16_dev, void* const* ys_fp16_dev, int n,
+                      int M, void* stream);
 
 /* Same map for callers whose activations live in HOST memory: copies x (host, [M][in]) to a
  * handle-owned staging buffer, runs bpdq_linear, copies y back to `y_fp16_host` and waits for

@@ -142,6 +142,26 @@ extern "C" int bpdq_linear_ex(bpdq_handle_t h, const void* x, void* y, int M, in
     }
 }
 
+extern "C" int bpdq_linear_batch(const bpdq_handle_t* hs, const void* const* xs, void* const* ys, int n, int M, void* stream) {
+    if (!hs || !xs || !ys) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: null array");
+    if (n < 1 || n > BPDQ_BATCH_MAX) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: n=%d outside [1, %d]", n, BPDQ_BATCH_MAX);
+    if (M < 0 || M > BPDQ_GEMV_MAX_M) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: M=%d outside [0, %d]", M, BPDQ_GEMV_MAX_M);
+    for (int k = 0; k < n; ++k) {
+        if (!hs[k]) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: null handle at %d", k);
+        if (M > hs[k]->max_M) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: M=%d exceeds max_M=%d of linear %d", M, hs[k]->max_M, k);
+        if (hs[k]->K != hs[0]->K || hs[k]->device != hs[0]->device)
+            return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: linear %d differs from linear 0 in K or device", k);
+        if (!gemv_supported(hs[k]->out, hs[k]->in, hs[k]->K, hs[k]->group))
+            return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear_batch: look-up-table kernel does not cover K=%d g=%d", hs[k]->K, hs[k]->group);
+        for (int j = 0; j < k; ++j)
+            if (hs[j] == hs[k]) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: handle %d repeats handle %d", k, j);
+        if (M > 0 && (!xs[k] || !ys[k] || !aligned16(xs[k]) || !aligned16(ys[k])))
+            return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: x and y of linear %d must be non-null and 16-byte aligned", k);
+    }
+    if (M == 0) return BPDQ_OK;
+    return launch_gemv_batch(hs, xs, ys, n, M, static_cast<cudaStream_t>(stream));
+}
+
 extern "C" int bpdq_linear(bpdq_handle_t h, const void* x, void* y, int M, void* stream) {
     return bpdq_linear_ex(h, x, y, M, BPDQ_KERNEL_AUTO, stream);
 }

@@ -41,17 +41,29 @@ constexpr int kChunkRgs = 8;                          // row groups (of 16 rows)
 constexpr int kMiscBytes = 4096;                      // xsum + completion list, at the start of shared memory
 constexpr int kMaxDone = 512;                         // completed chunks handled per batch
 
-struct GemvParams {
+// One linear of a launch.  A launch covers one or several linears (same K, same token count): their
+// (slice, row group) task spaces are concatenated and every CTA takes a contiguous share of the whole.
+struct GemvLinear {
     const uint8_t* blob;
     size_t planes_bytes;
     const __half* x;          // [MT][in]
     __half* y;                // [MT][out]
     float* ws;                // [MT][out] binary32 row sums, zero between calls
     unsigned* counters;       // [ceil(out/16 / kChunkRgs)] arrival counters, zero between calls
-    int* status;              // device status word
     int out, in, group;
     int nblocks, nslices, nrg;
-    int tasks_base, tasks_rem;   // task range of CTA b: b*base + min(b, rem), one longer for b < rem
+    int task_begin;           // first task of this linear in the concatenated task space
+};
+constexpr int kMaxBatch = BPDQ_BATCH_MAX;
+constexpr int kMaxGrid = 192;                        // CTAs of a launch (one per SM)
+// set-up and hand-over of one (slice, row range) segment, in tasks; measured optima for one / several linears per launch
+constexpr int kSegmentCostSingle = 32, kSegmentCostBatch = 48;
+
+struct GemvParams {
+    GemvLinear lin[kMaxBatch];
+    int n;                       // linears in this launch
+    int* status;                 // device status word
+    int t_begin[kMaxGrid + 1];   // CTA b takes the tasks [t_begin[b], t_begin[b+1]) of the concatenated space
     int dyn_smem;                // dynamic shared memory bytes of the launch
     int early_weights;           // the packed weights were complete before the preceding kernel of the stream started
 };
@@ -104,7 +116,7 @@ __device__ __forceinline__ float2 unpack2(unsigned long long v) {
 }
 
 template <int K, int MT, int D, int W>
-__global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p) {
+__global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_constant__ GemvParams p) {
     constexpr int kThreads = W * 32;
     constexpr int NS = K * MT;                        // look-up streams per step: (plane, token) pairs
     constexpr int NP = (NS + 1) / 2;                  // packed accumulators
@@ -138,18 +150,22 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
 #pragma unroll
     for (int s = 0; s < 16; ++s) off[s] = lut0 + 4u * ((s + a) & 15) + 64u * h;
 
-    // contiguous share of the (slice, row group) task space: base tasks each, the first `rem` CTAs one more
+    // contiguous share of the concatenated (linear, slice, row group) task space, cut by the host
     const int bid = blockIdx.x;
-    int t = bid * p.tasks_base + min(bid, p.tasks_rem);
-    const int t_end = t + p.tasks_base + (bid < p.tasks_rem ? 1 : 0);
-    const uint8_t* cbase = p.blob + p.planes_bytes;
-    const size_t plane_pitch = (size_t)p.out * 16;    // bytes between planes of one block
-    const size_t coef_pitch = (size_t)p.out * 2;      // bytes between coefficients of one group
+    int t = p.t_begin[bid];
+    const int t_end = p.t_begin[bid + 1];
+    int li = 0;                                       // linear that task t belongs to
 
     while (t < t_end) {
-        const int s = t / p.nrg;
-        const int rg_begin = t - s * p.nrg;
-        const int rg_end = min(p.nrg, rg_begin + (t_end - t));
+        while (li + 1 < p.n && t >= p.lin[li + 1].task_begin) ++li;
+        const GemvLinear& L = p.lin[li];
+        const uint8_t* cbase = L.blob + L.planes_bytes;
+        const size_t plane_pitch = (size_t)L.out * 16;    // bytes between planes of one block
+        const size_t coef_pitch = (size_t)L.out * 2;      // bytes between coefficients of one group
+        const int tl = t - L.task_begin;
+        const int s = tl / L.nrg;
+        const int rg_begin = tl - s * L.nrg;
+        const int rg_end = min(L.nrg, rg_begin + (t_end - t));
         const int ntask = (rg_end - rg_begin - wid + W - 1) / W;          // tasks of this warp (may be <= 0)
 
         // per-lane source pointers of the first task; a task further on is W*16 rows further on
@@ -161,11 +177,11 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 const int b = s * kSliceBlocks + 2 * q + h;
-                valid[q] = b < p.nblocks;                                  // false past the end of a ragged last slice
+                valid[q] = b < L.nblocks;                                  // false past the end of a ragged last slice
                 const int bb = valid[q] ? b : 0;
-                psrc[q] = p.blob + ((size_t)bb * K * p.out + r) * 16;
-                const int G = (bb * 128) / p.group;
-                csrc[q] = cbase + ((size_t)G * (K + 1) * p.out + r) * 2;
+                psrc[q] = L.blob + ((size_t)bb * K * L.out + r) * 16;
+                const int G = (bb * 128) / L.group;
+                csrc[q] = cbase + ((size_t)G * (K + 1) * L.out + r) * 2;
             }
         }
         auto load_task = [&](Task<K>& tk, int n) {
@@ -212,7 +228,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
         for (int m = 0; m < MT; ++m)
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                xraw[m][u] = col < p.in ? ldg_first4(p.x + (size_t)m * p.in + col + 8 * u) : 0u;
+                xraw[m][u] = col < L.in ? ldg_first4(L.x + (size_t)m * L.in + col + 8 * u) : 0u;
         if (!early) {
 #pragma unroll
             for (int d = 0; d < D; ++d)
@@ -316,7 +332,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
             if (h == 0) {
                 const int r = (rg_begin + wid + n * W) * 16 + a;
 #pragma unroll
-                for (int m = 0; m < MT; ++m) atomicAdd(&p.ws[(size_t)m * p.out + r], yacc[m]);
+                for (int m = 0; m < MT; ++m) atomicAdd(&L.ws[(size_t)m * L.out + r], yacc[m]);
             }
         };
         for (int n0 = 0; n0 < ntask; n0 += D) {
@@ -342,10 +358,10 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
             __syncthreads();
             for (int ck = ck0 + tid; ck < min(ck_end, ck0 + kMaxDone); ck += kThreads) {
                 const int lo = max(rg_begin, ck * kChunkRgs), hi = min(rg_end, (ck + 1) * kChunkRgs);
-                const int size = min(p.nrg, (ck + 1) * kChunkRgs) - ck * kChunkRgs;
-                const unsigned before = atomicAdd(&p.counters[ck], (unsigned)(hi - lo));
-                if (before + (unsigned)(hi - lo) == (unsigned)(size * p.nslices)) {
-                    p.counters[ck] = 0u;
+                const int size = min(L.nrg, (ck + 1) * kChunkRgs) - ck * kChunkRgs;
+                const unsigned before = atomicAdd(&L.counters[ck], (unsigned)(hi - lo));
+                if (before + (unsigned)(hi - lo) == (unsigned)(size * L.nslices)) {
+                    L.counters[ck] = 0u;
                     done[atomicAdd(ndone, 1)] = ck;
                 }
             }
@@ -358,9 +374,9 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const GemvParams p)
                     const int rem = idx % (kChunkRgs * 16 * MT);
                     const int m = rem / (kChunkRgs * 16);
                     const int r = ckd * kChunkRgs * 16 + rem % (kChunkRgs * 16);
-                    if (r < p.out) {
-                        float* src = p.ws + (size_t)m * p.out + r;
-                        p.y[(size_t)m * p.out + r] = __float2half_rn(__ldcg(src));
+                    if (r < L.out) {
+                        float* src = L.ws + (size_t)m * L.out + r;
+                        L.y[(size_t)m * L.out + r] = __float2half_rn(__ldcg(src));
                         __stcg(src, 0.f);
                     }
                 }
@@ -382,12 +398,64 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
         if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemv: shared memory opt-in: %s", cudaGetErrorString(e));
         configured_smem = smem;
     }
-    const long long total = (long long)p.nslices * p.nrg;
-    if (total >= (1ll << 31)) return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv: task space too large");
-    int grid = h->sm_count;
+    long long total = 0;
+    for (int k = 0; k < p.n; ++k) {
+        p.lin[k].task_begin = (int)total;
+        total += (long long)p.lin[k].nslices * p.lin[k].nrg;
+        if (total >= (1ll << 31)) return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv: task space too large");
+    }
+    // Cut the task space into one share per SM of equal cost, a segment (a CTA's visit to one slice
+    // of one linear: table set-up, hand-over) counting as kSegmentCost tasks.  Short slices (few
+    // output rows) would otherwise load the CTAs that get them with many set-ups.
+    int grid = h->sm_count < kMaxGrid ? h->sm_count : kMaxGrid;
     if ((long long)grid > total) grid = (int)total;
-    p.tasks_base = (int)(total / grid);
-    p.tasks_rem = (int)(total % grid);
+    {
+        const int kSegmentCost = p.n > 1 ? kSegmentCostBatch : kSegmentCostSingle;
+        long long nseg = 0;
+        for (int k = 0; k < p.n; ++k) nseg += p.lin[k].nslices;
+        // cost of the tasks [t0, t1) as one CTA's share
+        auto share_cost = [&](long long t0, long long t1) {
+            long long cost = 0;
+            int k = 0;
+            for (long long t = t0; t < t1;) {
+                while (k + 1 < p.n && t >= p.lin[k + 1].task_begin) ++k;
+                const long long in_slice = p.lin[k].nrg - (t - p.lin[k].task_begin) % p.lin[k].nrg;
+                const long long take = in_slice < t1 - t ? in_slice : t1 - t;
+                cost += kSegmentCost + take;
+                t += take;
+            }
+            return cost;
+        };
+        double target = (double)(total + nseg * kSegmentCost) / grid;
+        for (int round = 0; round < 8; ++round) {     // cuts inside slices add segments: raise the target until the last share fits
+            int b = 0, k = 0;
+            long long t = 0;                          // next unassigned task
+            p.t_begin[0] = 0;
+            double budget = target;
+            while (t < total && b < grid - 1) {
+                while (k + 1 < p.n && t >= p.lin[k + 1].task_begin) ++k;
+                const long long in_slice = p.lin[k].nrg - (t - p.lin[k].task_begin) % p.lin[k].nrg;   // tasks left in the current slice
+                if (budget < kSegmentCost + 8 && t > p.t_begin[b]) {         // not worth opening another segment here
+                    p.t_begin[++b] = (int)t;
+                    budget += target;
+                    continue;
+                }
+                budget -= kSegmentCost;
+                long long take = in_slice;
+                if ((double)take > budget) take = (long long)budget > 0 ? (long long)budget : 1;
+                t += take;
+                budget -= (double)take;
+                if (take < in_slice) {                                        // budget spent inside the slice
+                    p.t_begin[++b] = (int)t;
+                    budget += target;
+                }
+            }
+            for (int c = b + 1; c <= grid; ++c) p.t_begin[c] = (int)total;    // the last share takes what is left
+            const double last = (double)share_cost(p.t_begin[b], total);
+            if (last <= 1.05 * target) break;
+            target += (last - target) / grid;
+        }
+    }
     p.dyn_smem = smem;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid); cfg.blockDim = dim3(W * 32); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
@@ -408,15 +476,30 @@ int launch_one(bpdq_handle_s* h, const GemvParams& p, cudaStream_t stream) {
     return launch_cfg<K, MT, (K <= 2 ? 3 : 2), 16>(h, p, stream);
 }
 
+void fill_linear(GemvLinear& L, const bpdq_handle_s* h) {
+    L.blob = h->d_blob;
+    L.planes_bytes = h->planes_bytes;
+    L.ws = h->d_ws;
+    L.counters = h->d_counters;
+    L.out = h->out; L.in = h->in; L.group = h->group;
+    L.nblocks = h->in / 128;
+    L.nslices = (L.nblocks + kSliceBlocks - 1) / kSliceBlocks;
+    L.nrg = h->out / 16;
+    L.task_begin = 0;
+}
+
+// Passes of at most kMaxMT tokens over all linears of the batch.
 template <int K>
-int launch_k(bpdq_handle_s* h, GemvParams p, const __half* x, __half* y, int M, cudaStream_t stream) {
+int launch_k(bpdq_handle_s* const* hs, GemvParams p, const void* const* xs, void* const* ys, int M, cudaStream_t stream) {
     int m0 = 0;
     while (m0 < M) {
         int mt = M - m0;
         if (mt > kMaxMT) mt = kMaxMT;
-        p.x = x + (size_t)m0 * h->in;
-        p.y = y + (size_t)m0 * h->out;
-        const int rc = (mt == 1) ? launch_one<K, 1>(h, p, stream) : launch_one<K, 2>(h, p, stream);
+        for (int k = 0; k < p.n; ++k) {
+            p.lin[k].x = static_cast<const __half*>(xs[k]) + (size_t)m0 * hs[k]->in;
+            p.lin[k].y = static_cast<__half*>(ys[k]) + (size_t)m0 * hs[k]->out;
+        }
+        const int rc = (mt == 1) ? launch_one<K, 1>(hs[0], p, stream) : launch_one<K, 2>(hs[0], p, stream);
         if (rc != BPDQ_OK) return rc;
         m0 += mt;
     }
@@ -433,27 +516,28 @@ size_t gemv_workspace_bytes(int out, int, int, int, int, int) { return kMaxMT * 
 
 size_t gemv_counter_count(int out) { return ((size_t)out / 16 + kChunkRgs - 1) / kChunkRgs; }
 
-int launch_gemv(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
+int launch_gemv_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream) {
+    if (n < 1 || n > kMaxBatch) return set_error(BPDQ_ERR_INVALID, "gemv: %d linears in one launch (1..%d)", n, kMaxBatch);
     GemvParams p;
-    p.blob = h->d_blob;
-    p.planes_bytes = h->planes_bytes;
-    p.ws = h->d_ws;
-    p.counters = h->d_counters;
-    p.status = h->d_status;
-    p.early_weights = h->caller_blob ? 0 : 1;
-    p.out = h->out; p.in = h->in; p.group = h->group;
-    p.nblocks = h->in / 128;
-    p.nslices = (p.nblocks + kSliceBlocks - 1) / kSliceBlocks;
-    p.nrg = h->out / 16;
-    const __half* xp = static_cast<const __half*>(x);
-    __half* yp = static_cast<__half*>(y);
-    switch (h->K) {
-        case 1: return launch_k<1>(h, p, xp, yp, M, stream);
-        case 2: return launch_k<2>(h, p, xp, yp, M, stream);
-        case 3: return launch_k<3>(h, p, xp, yp, M, stream);
-        case 4: return launch_k<4>(h, p, xp, yp, M, stream);
-        default: return set_error(BPDQ_ERR_UNSUPPORTED, "gemv: K=%d", h->K);
+    p.n = n;
+    p.status = hs[0]->d_status;
+    p.early_weights = 1;
+    for (int k = 0; k < n; ++k) {
+        if (hs[k]->K != hs[0]->K) return set_error(BPDQ_ERR_INVALID, "gemv: linears of one launch must share K");
+        fill_linear(p.lin[k], hs[k]);
+        if (hs[k]->caller_blob) p.early_weights = 0;
     }
+    switch (hs[0]->K) {
+        case 1: return launch_k<1>(hs, p, xs, ys, M, stream);
+        case 2: return launch_k<2>(hs, p, xs, ys, M, stream);
+        case 3: return launch_k<3>(hs, p, xs, ys, M, stream);
+        case 4: return launch_k<4>(hs, p, xs, ys, M, stream);
+        default: return set_error(BPDQ_ERR_UNSUPPORTED, "gemv: K=%d", hs[0]->K);
+    }
+}
+
+int launch_gemv(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
+    return launch_gemv_batch(&h, &x, &y, 1, M, stream);
 }
 
 }  // namespace bpdq

@@ -59,6 +59,7 @@ int launch_fill(bpdq_handle_s* h, uint64_t seed, cudaStream_t stream);
 int launch_dequant(bpdq_handle_s* h, void* w, cudaStream_t stream);
 int launch_gemv_simple(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
 int launch_gemv(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
+int launch_gemv_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream);
 int launch_gemm(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
 size_t gemv_workspace_bytes(int out, int in, int K, int group, int max_M, int sm_count);
 size_t gemv_counter_count(int out);

@@ -1,0 +1,68 @@
+"""bpdq_linear_batch: several linears in one launch of the look-up-table kernel, against the checker."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2602_04163_b200 import binding, synth
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_batch(handles, xs_bits, M):
+    xs = [G.x_tensor(x) for x in xs_bits]
+    ys = [torch.full((M, h.out), float("nan"), dtype=torch.float16, device="cuda") for h in handles]
+    binding.bpdq_linear_batch(handles, [x.data_ptr() for x in xs], [y.data_ptr() for y in ys], M, G.stream_ptr())
+    torch.cuda.synchronize()
+    for h in handles:
+        h.bpdq_get_status(G.stream_ptr())
+    return [y.cpu().numpy().astype(np.float64) for y in ys]
+
+
+@pytest.mark.parametrize("K,M", [(2, 1), (3, 2), (2, 5), (1, 1)])
+def test_batch_matches_checker_and_single_launches(K, M):
+    import oracle
+    g = 128
+    shapes = [(160, 640), (48, 640), (272, 896), (16, 128), (1024, 2048)]     # ragged slices, tiny and multi-CTA linears
+    layers = [G.make_layer(90 + k, o, i, K, g, max_M=M) for k, (o, i) in enumerate(shapes)]
+    handles = [L[0] for L in layers]
+    x640 = synth.activations(91, M, 640)
+    xs = [x640, x640, synth.activations(92, M, 896), synth.activations(93, M, 128), synth.activations(94, M, 2048)]
+    for rep in range(2):                                                      # the second call finds the workspaces as the first left them
+        ys = _run_batch(handles, xs, M)
+        for (h, bits, coef), x, y in zip(layers, xs, ys):
+            y_ref, a_ref = oracle.linear(bits, coef, x, g)
+            G.assert_linear_close(y, y_ref, a_ref, f"batch rep {rep} {h.out}x{h.in_}")
+            y_single = G.run_linear(h, x, binding.KERNEL_GEMV)
+            assert np.allclose(y, y_single, rtol=2.0 ** -9, atol=1e-5)
+
+
+def test_batch_rejects_bad_arguments():
+    h1, _, _ = G.make_layer(1, 32, 128, 2, 128, max_M=2)
+    h2, _, _ = G.make_layer(2, 32, 128, 3, 128, max_M=2)
+    x = torch.zeros((2, 128), dtype=torch.float16, device="cuda")
+    y1 = torch.zeros((2, 32), dtype=torch.float16, device="cuda")
+    y2 = torch.zeros((2, 32), dtype=torch.float16, device="cuda")
+    n0 = h1.bpdq_launch_count()
+    for handles, M in (([h1, h1], 1), ([h1, h2], 1), ([h1], 3), ([h1] * 0, 1)):
+        with pytest.raises(binding.BpdqError) as ei:
+            binding.bpdq_linear_batch(handles, [x.data_ptr()] * len(handles), [y1.data_ptr(), y2.data_ptr()][:len(handles)], M,
+                                      G.stream_ptr())
+        assert ei.value.code == binding.ERR_INVALID
+    assert h1.bpdq_launch_count() == n0
+    binding.bpdq_linear_batch([h1], [0], [0], 0, G.stream_ptr())              # M = 0: nothing to do
+
+
+def test_batch_full_layer_sampled():
+    """All seven linears of a 72B-shaped layer (K = 2) in one launch; sampled rows against the checker."""
+    import oracle
+    K, g = 2, 128
+    shapes = synth.QWEN25_72B_LAYER
+    handles = [binding.Handle(o, i, K, g, None, 300 + li, 1) for li, (_, o, i) in enumerate(shapes)]
+    xb = {8192: synth.activations(301, 1, 8192), 29568: synth.activations(302, 1, 29568)}
+    ys = _run_batch(handles, [xb[i] for _, _, i in shapes], 1)
+    for li, ((name, o, i), y) in enumerate(zip(shapes, ys)):
+        rows = np.unique(np.concatenate([np.arange(0, o, max(1, o // 24)), [0, 15, 16, o - 16, o - 1]]))
+        y_ref, a_ref = oracle.linear(synth.plane_bits(300 + li, o, i, K, rows), synth.coefficients(300 + li, o, i, K, g, rows), xb[i], g)
+        G.assert_linear_close(y[:, rows], y_ref, a_ref, name)
+        assert np.all(np.isfinite(y))
