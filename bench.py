@@ -38,6 +38,9 @@ UNIT = "GB/s"
 GROUP = 128
 HBM_NOMINAL_GBS = 8000.0
 FALLBACK_HBM_GBS, FALLBACK_TFLOPS = 6650.0, 1590.0
+# dram__bytes_read.sum + dram__bytes_write.sum of the headline launch, from one ncu capture of this kernel as it stands
+# (set to None whenever the kernel changes until the counters are taken again)
+GEMV_TRAFFIC_BYTES_PER_LAUNCH = 265_048_832
 
 
 def useful_bytes(out: int, in_: int, K: int, g: int, M: int) -> int:
@@ -289,7 +292,7 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
             "gpu_launches": n_launch, "clocks": clocks,
             "roofline": {"bound": "hbm", "kernel": "gemv_lut_kernel", "achieved": per_gpu, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": per_gpu / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                         "frac_of_nominal_8tbs": per_gpu / HBM_NOMINAL_GBS, "traffic": None,
+                         "frac_of_nominal_8tbs": per_gpu / HBM_NOMINAL_GBS, "traffic": GEMV_TRAFFIC_BYTES_PER_LAUNCH,
                          "launches_per_step": 1, "algorithmic_bytes_per_launch": bytes_step}}
 
     # the same layer as seven separate bpdq_linear calls
