@@ -163,6 +163,21 @@ def run_reference(args, rank: int):
 # ------------------------------------------------------------------------------------------------
 # CUDA arm
 # ------------------------------------------------------------------------------------------------
+def slowest_rank(times_ms, world: int, device: str):
+    """Max over ranks of each timing (the job is as slow as its slowest replica); identity for one rank."""
+    import torch
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def replica_throughput_gbs(bytes_per_step: int, steps: int, world: int, ms_slowest: float) -> float:
+    """Whole-job rate of `world` independent replicas: all their bytes over the slowest rank's time."""
+    return world * bytes_per_step * steps / (ms_slowest * 1e-3) / 1e9
+
+
 class Layer:
     """Handles of one decoder layer's linears, generated on the device from a seed."""
 
@@ -270,13 +285,10 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
-    times = torch.tensor([ms_total, e2e_s * 1e3], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = float(times[0]), float(times[1])
+    ms_total, e2e_ms = slowest_rank([ms_total, e2e_s * 1e3], world, "cuda")
     bytes_step = layer_bytes(shapes, K, M)
-    value = world * bytes_step * args.steps / (ms_total * 1e-3) / 1e9
-    e2e_value = world * bytes_step * args.steps / (e2e_ms * 1e-3) / 1e9
+    value = replica_throughput_gbs(bytes_step, args.steps, world, ms_total)
+    e2e_value = replica_throughput_gbs(bytes_step, args.steps, world, e2e_ms)
     per_gpu = value / world
     n_launch = (launches2 - launches1)
 
