@@ -53,16 +53,36 @@ def test_batch_rejects_bad_arguments():
     binding.bpdq_linear_batch([h1], [0], [0], 0, G.stream_ptr())              # M = 0: nothing to do
 
 
-def test_batch_full_layer_sampled():
-    """All seven linears of a 72B-shaped layer (K = 2) in one launch; sampled rows against the checker."""
+@pytest.mark.parametrize("model,K", [("72b", 2), ("72b", 3), ("7b", 2)])
+def test_batch_full_layer_sampled(model, K):
+    """All seven linears of a Qwen2.5-shaped layer in one launch (the benchmark's step); sampled rows against the checker."""
     import oracle
-    K, g = 2, 128
-    shapes = synth.QWEN25_72B_LAYER
+    g = 128
+    shapes = synth.QWEN25_72B_LAYER if model == "72b" else synth.QWEN25_7B_LAYER
     handles = [binding.Handle(o, i, K, g, None, 300 + li, 1) for li, (_, o, i) in enumerate(shapes)]
-    xb = {8192: synth.activations(301, 1, 8192), 29568: synth.activations(302, 1, 29568)}
+    xb = {i: synth.activations(301 + i, 1, i) for i in sorted({i for _, _, i in shapes})}
     ys = _run_batch(handles, [xb[i] for _, _, i in shapes], 1)
     for li, ((name, o, i), y) in enumerate(zip(shapes, ys)):
         rows = np.unique(np.concatenate([np.arange(0, o, max(1, o // 24)), [0, 15, 16, o - 16, o - 1]]))
         y_ref, a_ref = oracle.linear(synth.plane_bits(300 + li, o, i, K, rows), synth.coefficients(300 + li, o, i, K, g, rows), xb[i], g)
         G.assert_linear_close(y[:, rows], y_ref, a_ref, name)
         assert np.all(np.isfinite(y))
+    for h in handles:
+        h.bpdq_destroy()
+
+
+@pytest.mark.parametrize("name,out,in_,K", [("gate", 29568, 8192, 2), ("down", 8192, 29568, 3)])
+def test_token_sweep_through_the_dispatcher(name, out, in_, K):
+    """M = 1..64 on 72B-shaped projections through bpdq_linear (look-up-table kernel below the threshold,
+    tensor-core kernel above); sampled rows against the checker."""
+    import oracle
+    g = 128
+    h = binding.Handle(out, in_, K, g, None, 400 + K, 64)
+    rows = np.unique(np.concatenate([np.arange(0, out, out // 12), [0, 127, 128, out - 1]]))
+    bits, coef = synth.plane_bits(400 + K, out, in_, K, rows), synth.coefficients(400 + K, out, in_, K, g, rows)
+    for M in (1, 2, 4, 8, 16, 32, 64):
+        x = synth.activations(500 + M, M, in_)
+        y = G.run_linear(h, x, binding.KERNEL_AUTO)
+        y_ref, a_ref = oracle.linear(bits, coef, x, g)
+        G.assert_linear_close(y[:, rows], y_ref, a_ref, f"{name} M={M}")
+    h.bpdq_destroy()
