@@ -56,7 +56,11 @@ template <int K, int BN> struct Cfg {
     static constexpr int kCoefBytes = (K + 1) * BM * 2;         // K+1 segments of 128 rows x 2 bytes
     static constexpr int kPackedBytes = (kPlaneBytes + kCoefBytes + 1023) / 1024 * 1024;
     static constexpr int kStageBytes = kATileBytes + kBTileBytes + kPackedBytes;
-    static constexpr int kStages = (222 * 1024) / kStageBytes > 8 ? 8 : (222 * 1024) / kStageBytes;
+    // Few tokens (BN <= 64): the kernel is bound by the decode threads, not by the MMAs, so two CTAs share an SM
+    // (half the shared memory each) and a 72B-shaped projection's row tiles run in one wave.
+    static constexpr int kCtasPerSm = BN <= 64 ? 2 : 1;
+    static constexpr int kSmemBudget = kCtasPerSm == 2 ? 110 * 1024 : 222 * 1024;
+    static constexpr int kStages = kSmemBudget / kStageBytes > 8 ? 8 : kSmemBudget / kStageBytes;
     static constexpr int kTmemCols = BN < 32 ? 32 : BN;        // power of two >= 32
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
 };
@@ -157,7 +161,7 @@ __host__ __device__ constexpr unsigned instr_desc_f16(int m, int n) {
 }
 
 template <int K, int BN>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, Cfg<K, BN>::kCtasPerSm)
 gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
     using C = Cfg<K, BN>;
     constexpr int S = C::kStages;
