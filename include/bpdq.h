@@ -136,7 +136,8 @@ BPDQ_API int bpdq_linear_ex(bpdq_handle_t h, const void* x_fp16_dev, void* y_fp1
  * BPDQ_KERNEL_GEMV computes it; the task spaces of the n linears are concatenated, so launch
  * ramp, table set-up and tail are paid once instead of n times.  hs, xs, ys are HOST arrays of n
  * handles / device pointers (read before the call returns); 1 <= n <= BPDQ_BATCH_MAX; the
- * handles are distinct, live on the current device, share K and have group 128 or 256;
+ * handles are distinct, live on the current device, share K, and either all or none of them
+ * have group 64;
  * 0 <= M <= min(max_M of every handle, BPDQ_GEMV_MAX_M).  Inputs may be shared between
  * linears; outputs must not overlap anything else.  BPDQ_ERR_INVALID / BPDQ_ERR_UNSUPPORTED
  * otherwise, with nothing launched. */
@@ -162,7 +163,7 @@ BPDQ_API int bpdq_linear_host(bpdq_handle_t h, const void* x_fp16_host, void* y_
  * status word) is a static device array inside the library, about 0.5 MB, held by every GPU
  * that loads the library until the process exits; it bounds the layer at
  * out <= BPDQ_NOALLOC_MAX_OUT rows (larger: BPDQ_ERR_INVALID, nothing is launched).  Shapes as
- * for bpdq_create, with group 128 or 256.
+ * for bpdq_create.
  *
  * The first call on a device looks up the array's device address and two device attributes;
  * make that first call outside any stream capture.  No call allocates or frees device or host

@@ -154,6 +154,8 @@ extern "C" int bpdq_linear_batch(const bpdq_handle_t* hs, const void* const* xs,
         if (M > hs[k]->max_M) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: M=%d exceeds max_M=%d of linear %d", M, hs[k]->max_M, k);
         if (hs[k]->K != hs[0]->K || hs[k]->device != hs[0]->device)
             return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: linear %d differs from linear 0 in K or device", k);
+        if ((hs[k]->group == 64) != (hs[0]->group == 64))
+            return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: linear %d and linear 0 differ in having group 64", k);
         if (!gemv_supported(hs[k]->out, hs[k]->in, hs[k]->K, hs[k]->group))
             return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear_batch: look-up-table kernel does not cover K=%d g=%d", hs[k]->K, hs[k]->group);
         for (int j = 0; j < k; ++j)

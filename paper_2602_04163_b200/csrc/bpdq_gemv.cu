@@ -70,10 +70,10 @@ struct GemvParams {
 
 // Registers of one task (16 rows x 4 blocks) of a lane: K plane units and K+1 coefficients for
 // each of its two blocks.
-template <int K>
+template <int K, int NG>
 struct Task {
     uint4 pl[2][K];
-    unsigned short cf[2][K + 1];
+    unsigned short cf[2][NG][K + 1];     // NG coefficient groups per 128-column block (two when g = 64)
 };
 
 __device__ __forceinline__ uint4 ldg_stream16(const uint8_t* p) {
@@ -115,11 +115,12 @@ __device__ __forceinline__ float2 unpack2(unsigned long long v) {
     return f;
 }
 
-template <int K, int MT, int D, int W>
+template <int K, int MT, int D, int W, bool G64>
 __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_constant__ GemvParams p) {
     constexpr int kThreads = W * 32;
     constexpr int NS = K * MT;                        // look-up streams per step: (plane, token) pairs
     constexpr int NP = (NS + 1) / 2;                  // packed accumulators
+    constexpr int NG = G64 ? 2 : 1;                   // coefficient groups per block
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int h = lane >> 4, a = lane & 15;
@@ -139,7 +140,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
         if (tid == 0) atomicExch(p.status, BPDQ_ERR_UNSUPPORTED);
         return;                                                          // uniform: no barrier has been reached
     }
-    float* xsum = reinterpret_cast<float*>(smem);                         // [MT][kSliceBlocks]
+    float* xsum = reinterpret_cast<float*>(smem);                         // [MT][kSliceBlocks][2]: per 64-column half block
     int* done = reinterpret_cast<int*>(smem + 64);                        // [kMaxDone]
     int* ndone = done + kMaxDone;
     float* lut = reinterpret_cast<float*>(smem + (lut0 - smem0));         // [MT][256][kSlots]
@@ -149,6 +150,10 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
     unsigned off[16];
 #pragma unroll
     for (int s = 0; s < 16; ++s) off[s] = lut0 + 4u * ((s + a) & 15) + 64u * h;
+    // steps at which this lane's chunk (logical byte (s + a) mod 16) lies in the block's first 64 columns
+    unsigned lo_steps = 0;
+#pragma unroll
+    for (int s = 0; s < 16; ++s) lo_steps |= (((s + a) & 15) < 8 ? 1u : 0u) << s;
 
     // contiguous share of the concatenated (linear, slice, row group) task space, cut by the host
     const int bid = blockIdx.x;
@@ -184,7 +189,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                 csrc[q] = cbase + ((size_t)G * (K + 1) * L.out + r) * 2;
             }
         }
-        auto load_task = [&](Task<K>& tk, int n) {
+        auto load_task = [&](Task<K, NG>& tk, int n) {
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 if (valid[q]) {
@@ -193,12 +198,16 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                     for (int i = 0; i < K; ++i) tk.pl[q][i] = ldg_stream16(ps + i * plane_pitch);
                     const uint8_t* cs = csrc[q] + (size_t)n * (W * 32);
 #pragma unroll
-                    for (int i = 0; i <= K; ++i) tk.cf[q][i] = ldg_stream2(cs + i * coef_pitch);
+                    for (int gg = 0; gg < NG; ++gg)
+#pragma unroll
+                        for (int i = 0; i <= K; ++i) tk.cf[q][gg][i] = ldg_stream2(cs + (gg * (K + 1) + i) * coef_pitch);
                 } else {                              // contributes nothing: zero planes, zero coefficients
 #pragma unroll
                     for (int i = 0; i < K; ++i) tk.pl[q][i] = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                    for (int i = 0; i <= K; ++i) tk.cf[q][i] = 0;
+                    for (int gg = 0; gg < NG; ++gg)
+#pragma unroll
+                        for (int i = 0; i <= K; ++i) tk.cf[q][gg][i] = 0;
                 }
             }
         };
@@ -212,7 +221,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
         const int col = s * (kSliceBlocks * 128) + (slot >> 2) * 32 + (slot & 3) * 2;
         // Before the first wait on the preceding kernel only the weights may be requested (they
         // belong to the handle and were complete long ago); then x, which that kernel may have written.
-        Task<K> tk[D];
+        Task<K, NG> tk[D];
         const bool early = !dep_waited && p.early_weights != 0;
         if (early) {
 #pragma unroll
@@ -261,16 +270,16 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
             }
         }
         __syncthreads();
-        if (tid < MT * kSliceBlocks) {
-            const int m = tid / kSliceBlocks, blk = tid % kSliceBlocks;
+        if (tid < MT * kSliceBlocks * 2) {            // sums of x over the two 64-column halves of every block
+            const int m = tid / (kSliceBlocks * 2), hb = tid % (kSliceBlocks * 2);
             float acc = 0.f;
-            for (int c = 0; c < 16; ++c) acc += lut[m * (kTableBytes / 4) + 255 * kSlots + blk * 16 + c];
-            xsum[m * kSliceBlocks + blk] = acc;
+            for (int c = 0; c < 8; ++c) acc += lut[m * (kTableBytes / 4) + 255 * kSlots + hb * 8 + c];
+            xsum[m * (kSliceBlocks * 2) + hb] = acc;
         }
         __syncthreads();
 
         // ---- stream the row groups of this slice ----
-        auto process_task = [&](const Task<K>& tk, int n) {
+        auto process_task = [&](const Task<K, NG>& tk, int n) {
             float yacc[MT];
 #pragma unroll
             for (int m = 0; m < MT; ++m) yacc[m] = 0.f;
@@ -282,6 +291,9 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
 #pragma unroll
                 for (int j = 0; j < NP; ++j) acc[j][0] = acc[j][1] = 0ull;
                 float held = 0.f;                     // odd stream count: the last stream pairs two steps
+                float Slo[NS];                        // g = 64: the part of every stream that falls into the block's first 64 columns
+#pragma unroll
+                for (int j = 0; j < NS; ++j) Slo[j] = 0.f;
 #pragma unroll
                 for (int st = 0; st < 16; ++st) {
                     float v[NS];
@@ -296,6 +308,10 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                             else if (q == 0) v[i * MT + m] = lds_table<kTableBytes>(addr);
                             else v[i * MT + m] = lds_table<kTableBytes + 128>(addr);
                         }
+                    }
+                    if (G64 && ((lo_steps >> st) & 1u)) {
+#pragma unroll
+                        for (int j = 0; j < NS; ++j) Slo[j] += v[j];
                     }
 #pragma unroll
                     for (int j = 0; j < NS / 2; ++j) add2(acc[j][st & 1], v[2 * j], v[2 * j + 1]);
@@ -316,14 +332,31 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                     S[NS - 1] = (e.x + e.y) + (o.x + o.y);
                 }
                 const int blk = 2 * q + h;
-                const float c0 = __half2float(__ushort_as_half(tk.cf[q][0]));
+                if (G64) {
+                    const float c0l = __half2float(__ushort_as_half(tk.cf[q][0][0]));
+                    const float c0h = __half2float(__ushort_as_half(tk.cf[q][NG - 1][0]));
 #pragma unroll
-                for (int m = 0; m < MT; ++m) yacc[m] = fmaf(c0, xsum[m * kSliceBlocks + blk], yacc[m]);
+                    for (int m = 0; m < MT; ++m)
+                        yacc[m] = fmaf(c0h, xsum[(m * kSliceBlocks + blk) * 2 + 1], fmaf(c0l, xsum[(m * kSliceBlocks + blk) * 2], yacc[m]));
 #pragma unroll
-                for (int i = 0; i < K; ++i) {
-                    const float ci = __half2float(__ushort_as_half(tk.cf[q][i + 1]));
+                    for (int i = 0; i < K; ++i) {
+                        const float cil = __half2float(__ushort_as_half(tk.cf[q][0][i + 1]));
+                        const float cih = __half2float(__ushort_as_half(tk.cf[q][NG - 1][i + 1]));
 #pragma unroll
-                    for (int m = 0; m < MT; ++m) yacc[m] = fmaf(ci, S[i * MT + m], yacc[m]);
+                        for (int m = 0; m < MT; ++m)
+                            yacc[m] = fmaf(cih, S[i * MT + m] - Slo[i * MT + m], fmaf(cil, Slo[i * MT + m], yacc[m]));
+                    }
+                } else {
+                    const float c0 = __half2float(__ushort_as_half(tk.cf[q][0][0]));
+#pragma unroll
+                    for (int m = 0; m < MT; ++m)
+                        yacc[m] = fmaf(c0, xsum[(m * kSliceBlocks + blk) * 2] + xsum[(m * kSliceBlocks + blk) * 2 + 1], yacc[m]);
+#pragma unroll
+                    for (int i = 0; i < K; ++i) {
+                        const float ci = __half2float(__ushort_as_half(tk.cf[q][0][i + 1]));
+#pragma unroll
+                        for (int m = 0; m < MT; ++m) yacc[m] = fmaf(ci, S[i * MT + m], yacc[m]);
+                    }
                 }
             }
             // the two half-warps hold the even-block and odd-block parts of the same 16 rows
@@ -387,14 +420,14 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
     }
 }
 
-template <int K, int MT, int D, int W>
+template <int K, int MT, int D, int W, bool G64>
 int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     static int configured_smem = 0;
     const int smem = 65536 + MT * kTableBytes;        // tables start at the first 64 KB boundary of the shared window
     if (smem > h->smem_optin)
         return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv: %d bytes of shared memory needed, device offers %d", smem, h->smem_optin);
     if (configured_smem != smem) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<K, MT, D, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<K, MT, D, W, G64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemv: shared memory opt-in: %s", cudaGetErrorString(e));
         configured_smem = smem;
     }
@@ -463,7 +496,7 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // lets this launch overlap the tail of the kernel before it
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_lut_kernel<K, MT, D, W>, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_lut_kernel<K, MT, D, W, G64>, p);
     h->launches += 1;
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemv launch: %s", cudaGetErrorString(e));
@@ -473,7 +506,8 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
 // Tasks kept in flight per lane: three while their registers fit (K <= 2), else two.
 template <int K, int MT>
 int launch_one(bpdq_handle_s* h, const GemvParams& p, cudaStream_t stream) {
-    return launch_cfg<K, MT, (K <= 2 ? 3 : 2), 16>(h, p, stream);
+    if (p.lin[0].group == 64) return launch_cfg<K, MT, (K <= 2 ? 2 : 1), 16, true>(h, p, stream);
+    return launch_cfg<K, MT, (K <= 2 ? 3 : 2), 16, false>(h, p, stream);
 }
 
 void fill_linear(GemvLinear& L, const bpdq_handle_s* h) {
@@ -510,7 +544,7 @@ int launch_k(bpdq_handle_s* const* hs, GemvParams p, const void* const* xs, void
 
 namespace bpdq {
 
-bool gemv_supported(int, int, int K, int group) { return K >= 1 && K <= 4 && (group == 128 || group == 256); }
+bool gemv_supported(int, int, int K, int group) { return K >= 1 && K <= 4 && (group == 64 || group == 128 || group == 256); }
 
 size_t gemv_workspace_bytes(int out, int, int, int, int, int) { return kMaxMT * (size_t)out * sizeof(float); }
 
@@ -524,6 +558,8 @@ int launch_gemv_batch(bpdq_handle_s* const* hs, const void* const* xs, void* con
     p.early_weights = 1;
     for (int k = 0; k < n; ++k) {
         if (hs[k]->K != hs[0]->K) return set_error(BPDQ_ERR_INVALID, "gemv: linears of one launch must share K");
+        if ((hs[k]->group == 64) != (hs[0]->group == 64))
+            return set_error(BPDQ_ERR_INVALID, "gemv: linears of one launch must all have group 64 or none of them");
         fill_linear(p.lin[k], hs[k]);
         if (hs[k]->caller_blob) p.early_weights = 0;
     }

@@ -45,6 +45,10 @@ def test_m_zero_and_bad_arguments():
     (2, 128, 272, 896, 4),       # 4 tokens = two passes of 2
     (3, 128, 144, 512, 7),       # 3 + 2 + 2
     (2, 128, 16, 128, 1),        # smallest supported shape
+    (2, 64, 80, 384, 1),         # a coefficient group per half block (the paper's W2-G64)
+    (3, 64, 272, 896, 2),        # W3-G64, two tokens
+    (4, 64, 48, 1536, 3),
+    (1, 64, 1024, 2048, 1),
 ])
 def test_lut_kernel(K, g, out, in_, M):
     h, bits, coef = G.make_layer(40 + K, out, in_, K, g, max_M=M)
