@@ -58,11 +58,14 @@ __device__ __forceinline__ void code_nibbles_word(const unsigned (&w)[K], unsign
 
 // The 2^K candidate values of one (row, group) (Eq. 7) with the decode rule's arithmetic: float(c0),
 // then "+ float(ci)" in binary32 for the set bits in plane order, one rounding to binary16.
-// Returned as byte tables for the byte-permute decode (K <= 3): lo[0] holds the low bytes of
-// candidates 0..3, lo[1] of candidates 4..7 (zero when K < 3); hi[] the high bytes.
+// Returned as byte tables for the byte-permute decode: lo[t] holds the low bytes of candidates
+// 4t..4t+3, hi[t] the high bytes (tables beyond 2^K candidates are zero); K = 4 uses all four.
+template <int K> struct ByteTables { unsigned lo[K == 4 ? 4 : 2], hi[K == 4 ? 4 : 2]; };
+
 template <int K>
-__device__ __forceinline__ void candidate_byte_tables(const float (&c)[K + 1], unsigned (&lo)[2], unsigned (&hi)[2]) {
-    static_assert(K >= 1 && K <= 3, "byte-permute decode covers at most eight candidates");
+__device__ __forceinline__ void candidate_byte_tables(const float (&c)[K + 1], ByteTables<K>& t) {
+    static_assert(K >= 1 && K <= 4, "at most sixteen candidates");
+    constexpr int NT = K == 4 ? 4 : 2;
     float acc[1 << K];
 #pragma unroll
     for (int code = 0; code < (1 << K); ++code) {
@@ -72,28 +75,50 @@ __device__ __forceinline__ void candidate_byte_tables(const float (&c)[K + 1], u
             if ((code >> i) & 1) a = __fadd_rn(a, c[i + 1]);
         acc[code] = a;
     }
-    unsigned pair[4] = {0u, 0u, 0u, 0u};             // candidates (2q, 2q+1) as two binary16 in one register
+    unsigned pair[2 * NT];                           // candidates (2q, 2q+1) as two binary16 in one register
 #pragma unroll
-    for (int q = 0; q < (1 << K) / 2 || q < 1; ++q) {
-        const __half2 h = __floats2half2_rn(acc[2 * q], (2 * q + 1) < (1 << K) ? acc[2 * q + 1] : 0.f);
+    for (int q = 0; q < 2 * NT; ++q) {
+        const __half2 h = __floats2half2_rn(2 * q < (1 << K) ? acc[(2 * q) & ((1 << K) - 1)] : 0.f,
+                                            2 * q + 1 < (1 << K) ? acc[(2 * q + 1) & ((1 << K) - 1)] : 0.f);
         pair[q] = *reinterpret_cast<const unsigned*>(&h);
     }
-    lo[0] = __byte_perm(pair[0], pair[1], 0x6420u);
-    hi[0] = __byte_perm(pair[0], pair[1], 0x7531u);
-    lo[1] = __byte_perm(pair[2], pair[3], 0x6420u);
-    hi[1] = __byte_perm(pair[2], pair[3], 0x7531u);
+#pragma unroll
+    for (int k = 0; k < NT; ++k) {
+        t.lo[k] = __byte_perm(pair[2 * k], pair[2 * k + 1], 0x6420u);
+        t.hi[k] = __byte_perm(pair[2 * k], pair[2 * k + 1], 0x7531u);
+    }
+}
+
+// Four binary16 values from the four code nibbles in the low half of `sel`.
+template <int K>
+__device__ __forceinline__ void decode4(const unsigned sel, const ByteTables<K>& t, unsigned& out01, unsigned& out23) {
+    unsigned l, h;
+    if constexpr (K == 4) {
+        // a byte-permute selects among eight bytes: candidates 0..7 and 8..15 are looked up separately
+        // (selector without its top bit) and the top bit of every code picks between the two results
+        const unsigned s7 = sel & 0x7777u;
+        unsigned m = (sel >> 3) & 0x1111u;                   // top bits at nibble positions 0, 4, 8, 12
+        m = (m & 0x0011u) | ((m & 0x1100u) << 8);            // ... at 0, 4, 16, 20
+        m = (m & 0x00010001u) | ((m & 0x00100010u) << 4);    // ... at 0, 8, 16, 24
+        m *= 0xFFu;                                          // one full byte per code
+        const unsigned la = __byte_perm(t.lo[0], t.lo[1], s7), lb = __byte_perm(t.lo[2], t.lo[3], s7);
+        const unsigned ha = __byte_perm(t.hi[0], t.hi[1], s7), hb = __byte_perm(t.hi[2], t.hi[3], s7);
+        l = (la & ~m) | (lb & m);
+        h = (ha & ~m) | (hb & m);
+    } else {
+        l = __byte_perm(t.lo[0], t.lo[1], sel);
+        h = __byte_perm(t.hi[0], t.hi[1], sel);
+    }
+    out01 = __byte_perm(l, h, 0x5140u);
+    out23 = __byte_perm(l, h, 0x7362u);
 }
 
 // Eight binary16 values (columns in order) from eight code nibbles.
-__device__ __forceinline__ uint4 decode8(const unsigned sel, const unsigned (&lo)[2], const unsigned (&hi)[2]) {
-    const unsigned sel_hi = __umulhi(sel, 0x10000u);         // sel >> 16 on the multiplier instead of the shifter
-    const unsigned l0 = __byte_perm(lo[0], lo[1], sel), h0 = __byte_perm(hi[0], hi[1], sel);
-    const unsigned l1 = __byte_perm(lo[0], lo[1], sel_hi), h1 = __byte_perm(hi[0], hi[1], sel_hi);
+template <int K>
+__device__ __forceinline__ uint4 decode8(const unsigned sel, const ByteTables<K>& t) {
     uint4 o;
-    o.x = __byte_perm(l0, h0, 0x5140u);
-    o.y = __byte_perm(l0, h0, 0x7362u);
-    o.z = __byte_perm(l1, h1, 0x5140u);
-    o.w = __byte_perm(l1, h1, 0x7362u);
+    decode4<K>(sel, t, o.x, o.y);
+    decode4<K>(__umulhi(sel, 0x10000u), t, o.z, o.w);        // sel >> 16 on the multiplier instead of the shifter
     return o;
 }
 

@@ -266,7 +266,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
         bool ok = true;
         for (int b = grp; b < nblocks && ok; b += kDecodeGroups) {
             unsigned cur[K][4];                          // logical words of this row's plane units
-            unsigned lo[2], hi[2];
+            bpdq::ByteTables<K> tab;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 const int kb = 2 * b + half;
@@ -292,7 +292,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
                         asm volatile("ld.shared.u16 %0, [%1];" : "=h"(hbits) : "r"(psrc + C::kPlaneBytes + i * (BM * 2) + rl * 2));
                         c[i] = __half2float(__ushort_as_half(hbits));
                     }
-                    bpdq::candidate_byte_tables<K>(c, lo, hi);
+                    bpdq::candidate_byte_tables<K>(c, tab);
                 }
                 const unsigned dst = a_base + s * kATileBytes;
 #pragma unroll
@@ -303,7 +303,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
                     bpdq::code_nibbles_word<K>(w, sel);
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        const uint4 v8 = bpdq::decode8(sel[u], lo, hi);
+                        const uint4 v8 = bpdq::decode8<K>(sel[u], tab);
                         asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + a_off[4 * wd + u]),
                                      "r"(v8.x), "r"(v8.y), "r"(v8.z), "r"(v8.w) : "memory");
                     }
@@ -405,7 +405,7 @@ int launch_k(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t strea
 namespace bpdq {
 
 bool gemm_supported(int, int, int K, int group) {
-    return K >= 1 && K <= 3 && (group == 64 || group == 128 || group == 256);
+    return K >= 1 && K <= 4 && (group == 64 || group == 128 || group == 256);
 }
 
 int launch_gemm(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
@@ -413,6 +413,7 @@ int launch_gemm(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t st
         case 1: return launch_k<1>(h, x, y, M, stream);
         case 2: return launch_k<2>(h, x, y, M, stream);
         case 3: return launch_k<3>(h, x, y, M, stream);
+        case 4: return launch_k<4>(h, x, y, M, stream);
         default: return set_error(BPDQ_ERR_UNSUPPORTED, "gemm: K=%d", h->K);
     }
 }

@@ -20,6 +20,8 @@ pytestmark = pytest.mark.gpu
     (3, 128, 384, 2048, 257),    # two token tiles of 256, the second holds one token
     (2, 128, 1024, 1024, 300),
     (2, 128, 128, 128, 1),       # a single token through the tensor-core path
+    (4, 128, 256, 512, 40),      # sixteen candidates per group (the paper's W4-G128): two byte-permutes and a select
+    (4, 64, 128, 384, 300),
 ])
 def test_gemm_kernel(K, g, out, in_, M):
     h, bits, coef = G.make_layer(60 + K, out, in_, K, g, max_M=M)
@@ -30,9 +32,10 @@ def test_gemm_kernel(K, g, out, in_, M):
     assert np.array_equal(y1, y2)                        # fixed accumulation order: bit-identical reruns
 
 
-def test_gemm_equals_dequant_times_x():
+@pytest.mark.parametrize("K", [1, 2, 3, 4])
+def test_gemm_equals_dequant_times_x(K):
     """The decoded operand is W^ itself: with one-hot tokens the kernel must return columns of bpdq_dequant exactly."""
-    K, g, out, in_ = 3, 128, 256, 512
+    g, out, in_ = 128, 256, 512
     h, bits, coef = G.make_layer(5, out, in_, K, g, max_M=in_)
     w = G.run_dequant(h).view(np.float16)
     x = np.eye(in_, dtype=np.float16)                    # token t selects column t
