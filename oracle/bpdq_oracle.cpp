@@ -27,8 +27,8 @@
 // bound, Proposition 1 (uniform grid as a special case, checked through an all-integer
 // route), all-zero / all-one plane closed forms, rounding ties and overflow, brute force on
 // tiny shapes against a differently structured decode, numpy's binary16 conversions, and a
-// float64 matrix product.  The acceptance bound on y (4e-3 * a + 1e-3) is stated by the
-// task, not by the paper: beyond that bound the y tolerance is "parity unpinned".
+// float64 matrix product.  The acceptance bound on y (4e-3 * a + 1e-3) is this library's
+// acceptance criterion, not a statement of the paper: beyond that bound the y tolerance is "parity unpinned".
 //
 // oracle_unpack is an independent reader of the device blob layout, written from the
 // layout's description (not from the library's packer):
