@@ -272,9 +272,12 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
           for in_ in xs}
     yh = {out: torch.empty((1, out), dtype=torch.float16).pin_memory() for out in ys}
 
+    yh_each = [torch.empty((1, o), dtype=torch.float16).pin_memory() for _, o, _ in shapes]
+    xh_ptrs = [xh[i].data_ptr() for _, _, i in shapes]
+    yh_ptrs = [y.data_ptr() for y in yh_each]
+
     def step_host(layer):
-        for (name, h) in layer.handles:
-            h.bpdq_linear_host(xh[h.in_].data_ptr(), yh[h.out].data_ptr(), M, sp)
+        binding.bpdq_linear_batch_host([h for _, h in layer.handles], xh_ptrs, yh_ptrs, M, sp)
 
     for w in range(max(3, args.warmup)):
         step_host(layers[w % copies])

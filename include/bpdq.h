@@ -144,6 +144,13 @@ BPDQ_API int bpdq_linear_ex(bpdq_handle_t h, const void* x_fp16_dev, void* y_fp1
 BPDQ_API int bpdq_linear_batch(const bpdq_handle_t* hs, const void* const* xs_fp16_dev, void* const* ys_fp16_dev, int n,
                       int M, void* stream);
 
+/* bpdq_linear_batch for callers whose activations live in HOST memory: copies every x[k] (host, [M][in_k]) to
+ * its handle's staging buffer, runs bpdq_linear_batch, copies every y[k] back to host memory and waits for
+ * the stream once.  Same argument rules as bpdq_linear_batch; pinned host memory keeps the copies
+ * asynchronous up to the final wait. */
+BPDQ_API int bpdq_linear_batch_host(const bpdq_handle_t* hs, const void* const* xs_fp16_host, void* const* ys_fp16_host, int n,
+                           int M, void* stream);
+
 /* Same map for callers whose activations live in HOST memory: copies x (host, [M][in]) to a
  * handle-owned staging buffer, runs bpdq_linear, copies y back to `y_fp16_host` and waits for
  * the stream.  Pinned host memory makes the copies asynchronous up to that wait. */

@@ -22,7 +22,7 @@ NOALLOC_MAX_OUT = 65536
 
 EXPORTS = ("bpdq_packed_bytes", "bpdq_pack", "bpdq_unpack", "bpdq_create", "bpdq_dequant", "bpdq_linear",
            "bpdq_linear_ex", "bpdq_linear_host", "bpdq_set_gemv_max_m", "bpdq_read_blob", "bpdq_get_status",
-           "bpdq_launch_count", "bpdq_destroy", "bpdq_last_error", "bpdq_linear_noalloc", "bpdq_linear_batch")
+           "bpdq_launch_count", "bpdq_destroy", "bpdq_last_error", "bpdq_linear_noalloc", "bpdq_linear_batch", "bpdq_linear_batch_host")
 
 _lib = None
 
@@ -52,6 +52,7 @@ def lib() -> ctypes.CDLL:
         L.bpdq_linear_ex.argtypes = [vp, vp, vp, i, i, vp]
         L.bpdq_linear_host.argtypes = [vp, vp, vp, i, vp]
         L.bpdq_linear_batch.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), i, i, vp]
+        L.bpdq_linear_batch_host.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), i, i, vp]
         L.bpdq_linear_noalloc.argtypes = [vp, i, i, i, i, vp, vp, i, vp]
         L.bpdq_set_gemv_max_m.argtypes = [vp, i]
         L.bpdq_read_blob.argtypes = [vp, vp]
@@ -122,6 +123,15 @@ def bpdq_linear_batch(handles, x_ptrs, y_ptrs, M: int, stream: int = 0) -> None:
         raise ValueError("handles, x_ptrs and y_ptrs must have the same length")
     arr = ctypes.c_void_p * n
     _check(lib().bpdq_linear_batch(arr(*[h._h for h in handles]), arr(*x_ptrs), arr(*y_ptrs), n, M, stream))
+
+
+def bpdq_linear_batch_host(handles, x_host_ptrs, y_host_ptrs, M: int, stream: int = 0) -> None:
+    """bpdq_linear_batch with host buffers: copies in, one launch, copies out, one wait."""
+    n = len(handles)
+    if not (n == len(x_host_ptrs) == len(y_host_ptrs)):
+        raise ValueError("handles, x_host_ptrs and y_host_ptrs must have the same length")
+    arr = ctypes.c_void_p * n
+    _check(lib().bpdq_linear_batch_host(arr(*[h._h for h in handles]), arr(*x_host_ptrs), arr(*y_host_ptrs), n, M, stream))
 
 
 class Handle:

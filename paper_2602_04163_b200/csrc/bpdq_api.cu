@@ -186,6 +186,36 @@ extern "C" int bpdq_linear_host(bpdq_handle_t h, const void* x_host, void* y_hos
     return BPDQ_OK;
 }
 
+extern "C" int bpdq_linear_batch_host(const bpdq_handle_t* hs, const void* const* xs_host, void* const* ys_host, int n, int M,
+                                      void* stream) {
+    if (!hs || !xs_host || !ys_host) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch_host: null array");
+    if (n < 1 || n > BPDQ_BATCH_MAX) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch_host: n=%d outside [1, %d]", n, BPDQ_BATCH_MAX);
+    for (int k = 0; k < n; ++k) {
+        if (!hs[k]) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch_host: null handle at %d", k);
+        if (M < 0 || M > hs[k]->max_M) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch_host: M=%d outside [0, max_M=%d] of linear %d", M, hs[k]->max_M, k);
+        if (M > 0 && (!xs_host[k] || !ys_host[k])) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch_host: null pointer at %d", k);
+    }
+    if (M == 0) return BPDQ_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const void* xd[BPDQ_BATCH_MAX];
+    void* yd[BPDQ_BATCH_MAX];
+    for (int k = 0; k < n; ++k) {
+        cudaError_t e = cudaMemcpyAsync(hs[k]->d_xstage, xs_host[k], (size_t)M * hs[k]->in * 2, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return cuda_fail("bpdq_linear_batch_host: copy in", e);
+        xd[k] = hs[k]->d_xstage;
+        yd[k] = hs[k]->d_ystage;
+    }
+    int rc = bpdq_linear_batch(hs, xd, yd, n, M, stream);
+    if (rc != BPDQ_OK) return rc;
+    for (int k = 0; k < n; ++k) {
+        cudaError_t e = cudaMemcpyAsync(ys_host[k], hs[k]->d_ystage, (size_t)M * hs[k]->out * 2, cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return cuda_fail("bpdq_linear_batch_host: copy out", e);
+    }
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail("bpdq_linear_batch_host: synchronize", e);
+    return BPDQ_OK;
+}
+
 extern "C" int bpdq_set_gemv_max_m(bpdq_handle_t h, int max_gemv_m) {
     if (!h) return set_error(BPDQ_ERR_INVALID, "bpdq_set_gemv_max_m: null handle");
     if (max_gemv_m < 0 || max_gemv_m > BPDQ_GEMV_MAX_M)

@@ -86,3 +86,17 @@ def test_token_sweep_through_the_dispatcher(name, out, in_, K):
         y_ref, a_ref = oracle.linear(bits, coef, x, g)
         G.assert_linear_close(y[:, rows], y_ref, a_ref, f"{name} M={M}")
     h.bpdq_destroy()
+
+
+def test_batch_host_buffers_match_device_call():
+    K, g, M = 2, 128, 2
+    shapes = [(160, 640), (48, 640), (272, 896)]
+    layers = [G.make_layer(190 + k, o, i, K, g, max_M=M) for k, (o, i) in enumerate(shapes)]
+    handles = [L[0] for L in layers]
+    xs = [synth.activations(191 + k, M, i) for k, (_, i) in enumerate(shapes)]
+    want = _run_batch(handles, xs, M)
+    xh = [torch.from_numpy(x.view(np.int16).copy()).view(torch.float16).pin_memory() for x in xs]
+    yh = [torch.full((M, o), float("nan"), dtype=torch.float16).pin_memory() for o, _ in shapes]
+    binding.bpdq_linear_batch_host(handles, [x.data_ptr() for x in xh], [y.data_ptr() for y in yh], M, G.stream_ptr())
+    for y, w in zip(yh, want):
+        assert np.allclose(y.numpy().astype(np.float64), w, rtol=2.0 ** -9, atol=1e-5)
