@@ -15,7 +15,7 @@
 // planes.  A warp takes 16 rows x 4 blocks per task: lane (h, a) = (lane/16, lane%16) owns row a
 // and the two blocks of parity h.  Its 16-byte plane units and binary16 coefficients come straight
 // from global memory into registers (16 lanes x 16 bytes = 256 contiguous bytes per request), two
-// or three tasks ahead, so that HBM latency is covered by loads in flight and shared memory
+// tasks ahead, so that HBM latency is covered by loads in flight and shared memory
 // carries nothing but the look-ups.  The blob stores, at byte p of row r, the 8-column chunk
 // ("logical byte") (p + r) mod 16, and table entries are laid out as [entry][slot],
 // slot = 16*block + chunk, so at every step the 32 lanes of a warp hit 32 different banks whatever
@@ -108,6 +108,17 @@ __device__ __forceinline__ unsigned word_of(const uint4& v, int k) {
 // A pair of binary32 accumulators in one 64-bit register: (lo, hi) += (a, b) as one packed add.
 __device__ __forceinline__ void add2(unsigned long long& acc, float a, float b) {
     asm("{\n\t.reg .b64 t;\n\tmov.b64 t, {%1, %2};\n\tadd.rn.f32x2 %0, %0, t;\n\t}" : "+l"(acc) : "f"(a), "f"(b));
+}
+// Two table look-ups and their packed add in one statement, so that the two loaded values are born as the
+// register pair the packed add reads (separate loads would each need a move into the pair).
+template <int IMM0, int IMM1>
+__device__ __forceinline__ void lookup2_add(unsigned long long& acc, unsigned addr0, unsigned addr1) {
+    asm("{\n\t.reg .f32 a, b;\n\t.reg .b64 t;\n\t"
+        "ld.shared.f32 a, [%1+%3];\n\t"
+        "ld.shared.f32 b, [%2+%4];\n\t"
+        "mov.b64 t, {a, b};\n\t"
+        "add.rn.f32x2 %0, %0, t;\n\t}"
+        : "+l"(acc) : "r"(addr0), "r"(addr1), "n"(IMM0), "n"(IMM1));
 }
 __device__ __forceinline__ float2 unpack2(unsigned long long v) {
     float2 f;
@@ -213,11 +224,13 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
         };
 
         // ---- this thread's inputs for the table build and the first tasks' weights ----
-        static_assert(kSlots * 8 == W * 32, "one table item (slot, entry block) per thread");
-        const int slot = tid & (kSlots - 1);          // chunk table
-        const int eh = tid >> 6;                      // entries eh*32 .. eh*32+31 share inputs 5..7
+        // table items (slot, entry block): kSlots * 8 of them, IT per thread; item = tid + it * kThreads,
+        // slot = item % 64 (chunk table), eh = item / 64 (entries eh*32 .. eh*32+31 share inputs 5..7).
         // slot = 16*block + logical byte L; L = 4k + q is byte q of 32-column word k, and bit
         // 4*jj + u of that byte is column 32k + 8u + 2q + jj: four pairs of adjacent inputs
+        static_assert((kSlots * 8) % (W * 32) == 0, "whole table items per thread");
+        constexpr int IT = kSlots * 8 / (W * 32);
+        const int slot = tid & (kSlots - 1);          // kThreads is a multiple of 64: the same slot for all of a thread's items
         const int col = s * (kSliceBlocks * 128) + (slot >> 2) * 32 + (slot & 3) * 2;
         // Before the first wait on the preceding kernel only the weights may be requested (they
         // belong to the handle and were complete long ago); then x, which that kernel may have written.
@@ -245,7 +258,9 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
         }
 
         // ---- build the 64 chunk tables of this slice (per token) ----
-        {
+#pragma unroll
+        for (int it = 0; it < IT; ++it) {
+            const int eh = (tid + it * kThreads) >> 6;
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
                 float xs[8];                          // xs[t]: the input that bit t of the plane byte selects
@@ -291,33 +306,58 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
 #pragma unroll
                 for (int j = 0; j < NP; ++j) acc[j][0] = acc[j][1] = 0ull;
                 float held = 0.f;                     // odd stream count: the last stream pairs two steps
+                unsigned held_addr = 0u;
                 float Slo[NS];                        // g = 64: the part of every stream that falls into the block's first 64 columns
 #pragma unroll
                 for (int j = 0; j < NS; ++j) Slo[j] = 0.f;
 #pragma unroll
                 for (int st = 0; st < 16; ++st) {
-                    float v[NS];
+                    // address = slot address with the plane byte in bits 8..15
+                    unsigned addr[K];
 #pragma unroll
-                    for (int i = 0; i < K; ++i) {
-                        // address = slot address with the plane byte in bits 8..15
-                        const unsigned addr = __byte_perm(word_of(tk.pl[q][i], st >> 2), off[st], 0x7604u | ((st & 3) << 4));
+                    for (int i = 0; i < K; ++i)
+                        addr[i] = __byte_perm(word_of(tk.pl[q][i], st >> 2), off[st], 0x7604u | ((st & 3) << 4));
+                    constexpr int QI = 128;               // the block pair and the token's table go into the immediate
+                    if constexpr (G64) {
+                        float v[NS];
 #pragma unroll
-                        for (int m = 0; m < MT; ++m) {      // the token's table and the block pair go into the immediate
-                            if (m == 0 && q == 0) v[i * MT + m] = lds_table<0>(addr);
-                            else if (m == 0) v[i * MT + m] = lds_table<128>(addr);
-                            else if (q == 0) v[i * MT + m] = lds_table<kTableBytes>(addr);
-                            else v[i * MT + m] = lds_table<kTableBytes + 128>(addr);
+                        for (int i = 0; i < K; ++i)
+#pragma unroll
+                            for (int m = 0; m < MT; ++m) {
+                                if (m == 0 && q == 0) v[i * MT + m] = lds_table<0>(addr[i]);
+                                else if (m == 0) v[i * MT + m] = lds_table<QI>(addr[i]);
+                                else if (q == 0) v[i * MT + m] = lds_table<kTableBytes>(addr[i]);
+                                else v[i * MT + m] = lds_table<kTableBytes + QI>(addr[i]);
+                            }
+                        if ((lo_steps >> st) & 1u) {
+#pragma unroll
+                            for (int j = 0; j < NS; ++j) Slo[j] += v[j];
                         }
-                    }
-                    if (G64 && ((lo_steps >> st) & 1u)) {
 #pragma unroll
-                        for (int j = 0; j < NS; ++j) Slo[j] += v[j];
-                    }
+                        for (int j = 0; j < NS / 2; ++j) add2(acc[j][st & 1], v[2 * j], v[2 * j + 1]);
+                        if (NS & 1) {
+                            if ((st & 1) == 0) held = v[NS - 1];
+                            else add2(acc[NP - 1][(st >> 1) & 1], held, v[NS - 1]);
+                        }
+                    } else if constexpr (MT == 2) {
+                        // pair = the two tokens of one plane: one address, two tables
 #pragma unroll
-                    for (int j = 0; j < NS / 2; ++j) add2(acc[j][st & 1], v[2 * j], v[2 * j + 1]);
-                    if (NS & 1) {
-                        if ((st & 1) == 0) held = v[NS - 1];
-                        else add2(acc[NP - 1][(st >> 1) & 1], held, v[NS - 1]);
+                        for (int i = 0; i < K; ++i) {
+                            if (q == 0) lookup2_add<0, kTableBytes>(acc[i][st & 1], addr[i], addr[i]);
+                            else lookup2_add<QI, kTableBytes + QI>(acc[i][st & 1], addr[i], addr[i]);
+                        }
+                    } else {
+                        // one token: pair = two planes; an odd plane left over pairs two consecutive steps
+#pragma unroll
+                        for (int j = 0; j < K / 2; ++j) {
+                            if (q == 0) lookup2_add<0, 0>(acc[j][st & 1], addr[2 * j], addr[2 * j + 1]);
+                            else lookup2_add<QI, QI>(acc[j][st & 1], addr[2 * j], addr[2 * j + 1]);
+                        }
+                        if (K & 1) {
+                            if ((st & 1) == 0) held_addr = addr[K - 1];
+                            else if (q == 0) lookup2_add<0, 0>(acc[NP - 1][(st >> 1) & 1], held_addr, addr[K - 1]);
+                            else lookup2_add<QI, QI>(acc[NP - 1][(st >> 1) & 1], held_addr, addr[K - 1]);
+                        }
                     }
                 }
                 float S[NS];
@@ -503,11 +543,12 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     return BPDQ_OK;
 }
 
-// Tasks kept in flight per lane: three while their registers fit (K <= 2), else two.
+// Tasks kept in flight per lane: two (a third costs more in recomputed addresses than it hides in latency);
+// one when the second coefficient group of g = 64 takes the registers (K >= 3).
 template <int K, int MT>
 int launch_one(bpdq_handle_s* h, const GemvParams& p, cudaStream_t stream) {
     if (p.lin[0].group == 64) return launch_cfg<K, MT, (K <= 2 ? 2 : 1), 16, true>(h, p, stream);
-    return launch_cfg<K, MT, (K <= 2 ? 3 : 2), 16, false>(h, p, stream);
+    return launch_cfg<K, MT, 2, 16, false>(h, p, stream);
 }
 
 void fill_linear(GemvLinear& L, const bpdq_handle_s* h) {
