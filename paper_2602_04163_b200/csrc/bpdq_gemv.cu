@@ -161,6 +161,8 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
     unsigned off[16];
 #pragma unroll
     for (int s = 0; s < 16; ++s) off[s] = lut0 + 4u * ((s + a) & 15) + 64u * h;
+#pragma unroll
+    for (int s = 0; s < 16; ++s) asm volatile("" : "+r"(off[s]));   // opaque: kept in registers instead of being recomputed at every use
     // steps at which this lane's chunk (logical byte (s + a) mod 16) lies in the block's first 64 columns
     unsigned lo_steps = 0;
 #pragma unroll
