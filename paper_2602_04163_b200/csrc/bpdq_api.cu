@@ -64,10 +64,9 @@ extern "C" int bpdq_create(bpdq_handle_t* hp, int out, int in, int K, int group,
     h->blob_bytes = h->planes_bytes + coefs_bytes(out, in, K, group);
     h->ws_bytes = gemv_workspace_bytes(out, in, K, group, max_M, h->sm_count);
     h->n_counters = gemv_counter_count(out);
-    // Measured crossover on 72B-shaped layers: with at least one 128-row tile per SM the tensor-core kernel
-    // (two CTAs per SM below 65 tokens) wins from M = 5; a layer with few output rows leaves it most of the
-    // SMs idle and two-token passes of the look-up-table kernel stay ahead up to M = 12.
-    h->gemv_max_m = (out + 127) / 128 >= h->sm_count ? 4 : 12;
+    // Measured crossover on 72B-shaped layers: two two-token passes of the look-up-table kernel (about 75 us on
+    // the largest projections) still beat the tensor-core kernel (86-94 us up to 64 tokens), a third pass does not.
+    h->gemv_max_m = 4;
 
     const size_t stage_x = (size_t)max_M * in * 2, stage_y = (size_t)max_M * out * 2;
     if ((e = cudaMalloc(&h->d_blob, h->blob_bytes)) != cudaSuccess ||

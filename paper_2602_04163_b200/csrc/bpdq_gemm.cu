@@ -71,6 +71,11 @@ struct GemmParams {
     __half* y;                // [M][out]
     int* status;
     int out, in, group, M;
+    // split over the input dimension (few tokens, fewer row tiles than SMs): gridDim.z CTAs share an output tile,
+    // each takes kb_per stages, adds its partial tile into `ws` and the last to arrive writes y
+    int kb_per;               // stages per CTA (even: a 128-column block is never cut)
+    float* ws;                // [M][out] binary32, zero between calls (only used when gridDim.z > 1)
+    unsigned* counters;       // one arrival counter per 128-row tile, zero between calls
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -183,7 +188,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int row0 = blockIdx.x * BM;          // first output row of this CTA
     const int tok0 = blockIdx.y * BN;          // first token of this CTA
-    const int nkb = p.in / BK;
+    const int kb0 = blockIdx.z * p.kb_per;           // this CTA's stages: [kb0, kb1) of the in / 64 stages of the row
+    const int kb1 = min(p.in / BK, kb0 + p.kb_per);
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
@@ -211,9 +217,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
             const int nrows = min(BM, p.out - row0);     // ragged last row tile: a multiple of 16
             const unsigned seg_p = (unsigned)nrows * 16u, seg_c = (unsigned)nrows * 2u;
             const uint8_t* cbase = p.blob + p.planes_bytes;
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % S;
-                const unsigned ph = (unsigned)(kb / S) & 1u;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                const int s = (kb - kb0) % S;
+                const unsigned ph = (unsigned)((kb - kb0) / S) & 1u;
                 if (!mbar_wait(empty(s), ph ^ 1u, abort_flag, p.status)) break;
                 // packed operands first: the decode threads are the longer leg of the pipeline
                 const bool first_half = (kb & 1) == 0;   // the block's plane units travel with its first stage
@@ -237,9 +243,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
         if (lane == 0) {
             constexpr unsigned idesc = instr_desc_f16(BM, BN);
             bool ok = true;
-            for (int kb = 0; kb < nkb && ok; ++kb) {
-                const int s = kb % S;
-                const unsigned ph = (unsigned)(kb / S) & 1u;
+            for (int kb = kb0; kb < kb1 && ok; ++kb) {
+                const int s = (kb - kb0) % S;
+                const unsigned ph = (unsigned)((kb - kb0) / S) & 1u;
                 ok = mbar_wait(full_a(s), ph, abort_flag, p.status) && mbar_wait(full_b(s), ph, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
@@ -247,7 +253,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
                 const uint64_t bdesc = smem_desc_sw128(b_base + s * C::kBTileBytes);
 #pragma unroll
                 for (int k4 = 0; k4 < BK / 16; ++k4)     // 16 columns = 32 bytes further along the swizzled row
-                    umma_f16(tmem_d, adesc + 2u * k4, bdesc + 2u * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+                    umma_f16(tmem_d, adesc + 2u * k4, bdesc + 2u * k4, idesc, ((kb - kb0) | k4) != 0 ? 1u : 0u);
                 umma_commit(empty(s));                   // frees the stage once these MMAs have read it
             }
             umma_commit(acc_full);                       // arrives when every MMA above has completed
@@ -259,19 +265,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
         const int rl = quad * 32 + lane;                 // row inside the tile
         const int r = row0 + rl;
         const bool row_ok = r < p.out;                   // rows past a ragged last tile decode stale bytes; nothing of theirs is stored
-        const int nblocks = p.in / 128;
         unsigned a_off[8];                               // swizzled byte offset of each 16-byte chunk of this thread's row
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) a_off[ch] = (unsigned)rl * 128u + (((unsigned)ch ^ (unsigned)(rl & 7)) << 4);
         bool ok = true;
-        for (int b = grp; b < nblocks && ok; b += kDecodeGroups) {
+        for (int b = kb0 / 2 + grp; 2 * b < kb1 && ok; b += kDecodeGroups) {
             unsigned cur[K][4];                          // logical words of this row's plane units
             bpdq::ByteTables<K> tab;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 const int kb = 2 * b + half;
-                const int s = kb % S;
-                const unsigned ph = (unsigned)(kb / S) & 1u;
+                const int s = (kb - kb0) % S;
+                const unsigned ph = (unsigned)((kb - kb0) / S) & 1u;
                 if (!mbar_wait(full_p(s), ph, abort_flag, p.status)) { ok = false; break; }
                 const unsigned psrc = p_base + s * C::kPackedBytes;
                 if (half == 0) {
@@ -326,17 +331,43 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const int t = tok0 + c0 + j;
-                        if (t < p.M) p.y[(size_t)t * p.out + r] = __float2half_rn(__uint_as_float(v[j]));
+                        if (t < p.M) {
+                            if (gridDim.z > 1) atomicAdd(p.ws + (size_t)t * p.out + r, __uint_as_float(v[j]));
+                            else p.y[(size_t)t * p.out + r] = __float2half_rn(__uint_as_float(v[j]));
+                        }
                     }
                 }
             }
         }
     }
+    if (gridDim.z > 1) __threadfence();              // this thread's partial sums are out before the tile's counter moves
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_d, C::kTmemCols);
+    }
+    if (gridDim.z > 1) {
+        // the last of the CTAs that share this output tile rounds it to binary16, writes y and zeroes the workspace
+        int* last = reinterpret_cast<int*>(const_cast<int*>(abort_flag)) + 1;
+        if (tid == 0) {
+            const unsigned before = atomicAdd(p.counters + blockIdx.x, 1u);
+            *last = before == gridDim.z - 1;
+            if (*last) p.counters[blockIdx.x] = 0u;
+        }
+        __syncthreads();
+        if (*last) {
+            __threadfence();
+            const int ntok = min(BN, p.M - tok0);
+            for (int idx = tid; idx < ntok * BM; idx += kThreads) {
+                const int t = tok0 + idx / BM, r = row0 + idx % BM;
+                if (r < p.out) {
+                    float* src = p.ws + (size_t)t * p.out + r;
+                    p.y[(size_t)t * p.out + r] = __float2half_rn(__ldcg(src));
+                    __stcg(src, 0.f);
+                }
+            }
+        }
     }
 }
 
@@ -384,7 +415,21 @@ int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t st
     GemmParams p;
     p.blob = h->d_blob; p.planes_bytes = h->planes_bytes; p.y = static_cast<__half*>(y); p.status = h->d_status;
     p.out = h->out; p.in = h->in; p.group = h->group; p.M = M;
-    const dim3 grid((h->out + BM - 1) / BM, (M + BN - 1) / BN);
+    p.ws = h->d_ws; p.counters = h->d_counters;
+    dim3 grid((h->out + BM - 1) / BM, (M + BN - 1) / BN);
+    const int nkb = h->in / BK;
+    p.kb_per = nkb;
+    if (grid.y == 1 && (size_t)M * h->out * sizeof(float) <= h->ws_bytes) {
+        // fewer output tiles than CTA slots: split the input dimension so that every SM gets work
+        const int slots = h->sm_count * C::kCtasPerSm;
+        int splits = slots / (int)grid.x;
+        if (splits > 8) splits = 8;
+        if (splits > nkb / 16) splits = nkb / 16;     // at least 16 stages (1024 columns) per CTA
+        if (splits > 1) {
+            p.kb_per = ((nkb + splits - 1) / splits + 1) / 2 * 2;
+            grid.z = (nkb + p.kb_per - 1) / p.kb_per;
+        }
+    }
     gemm_kernel<K, BN><<<grid, kThreads, C::kSmemBytes, stream>>>(map, p);
     h->launches += 1;
     cudaError_t e = cudaGetLastError();

@@ -589,7 +589,12 @@ namespace bpdq {
 
 bool gemv_supported(int, int, int K, int group) { return K >= 1 && K <= 4 && (group == 64 || group == 128 || group == 256); }
 
-size_t gemv_workspace_bytes(int out, int, int, int, int, int) { return kMaxMT * (size_t)out * sizeof(float); }
+// binary32 row sums: kMaxMT tokens for the look-up-table kernel; up to 64 tokens for the tensor-core kernel's split
+// over the input dimension
+size_t gemv_workspace_bytes(int out, int, int, int, int max_M, int) {
+    const int tokens = max_M < kMaxMT ? kMaxMT : (max_M > 64 ? 64 : max_M);
+    return (size_t)tokens * out * sizeof(float);
+}
 
 size_t gemv_counter_count(int out) { return ((size_t)out / 16 + kChunkRgs - 1) / kChunkRgs; }
 

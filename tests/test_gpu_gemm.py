@@ -22,6 +22,9 @@ pytestmark = pytest.mark.gpu
     (2, 128, 128, 128, 1),       # a single token through the tensor-core path
     (4, 128, 256, 512, 40),      # sixteen candidates per group (the paper's W4-G128): two byte-permutes and a select
     (4, 64, 128, 384, 300),
+    (2, 128, 256, 4096, 40),     # few row tiles, long rows: four CTAs share an output tile (split over the input dimension)
+    (3, 64, 128, 8192, 64),      # eight-way split
+    (4, 128, 384, 2048, 7),      # two-way split, ragged token tile
 ])
 def test_gemm_kernel(K, g, out, in_, M):
     h, bits, coef = G.make_layer(60 + K, out, in_, K, g, max_M=M)
@@ -29,7 +32,10 @@ def test_gemm_kernel(K, g, out, in_, M):
     G.check_linear(h, bits, coef, x, g, binding.KERNEL_GEMM, what="gemm")
     y1 = G.run_linear(h, x, binding.KERNEL_GEMM)
     y2 = G.run_linear(h, x, binding.KERNEL_GEMM)
-    assert np.array_equal(y1, y2)                        # fixed accumulation order: bit-identical reruns
+    if M > 64 or in_ < 2048:
+        assert np.array_equal(y1, y2)                    # one CTA per output tile, fixed accumulation order: bit-identical reruns
+    else:                                                # CTAs that share a tile add their parts in a free order: last binary16 digit
+        assert np.allclose(y1, y2, rtol=2.0 ** -9, atol=1e-5)
 
 
 @pytest.mark.parametrize("K", [1, 2, 3, 4])
