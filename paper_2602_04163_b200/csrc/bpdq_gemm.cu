@@ -27,6 +27,10 @@
 // the token columns: tcgen05.ld gives a thread its output row for 16 tokens at a time; adjacent
 // threads hold adjacent output indices, so a warp writes 64 contiguous bytes of y per token.
 //
+// Two kernels share this scheme: gemm_kernel (one output tile per CTA; token tiles of 32..128, two CTAs per SM
+// and a split over the input dimension when tokens are few) and gemm_persistent_kernel (token tile 256: one
+// CTA per SM walks over tiles, two TMEM accumulators, separate epilogue warps; described at its definition).
+//
 // Pipeline: per stage four mbarriers -- full_b (x tile landed), full_p (planes and coefficients
 // landed; the producer issued them after `empty`, so the stage's A slot is free as well), full_a
 // (128 decode threads arrived after a proxy fence), empty (tcgen05.commit of the MMAs that read
@@ -371,6 +375,232 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
     }
 }
 
+// ---- persistent variant for many tokens (token tile 256) -------------------------------------------------
+// One CTA per SM walks over output tiles (row tile fastest, so that the CTAs running together share one
+// 256-token slab of x in L2).  TMEM holds two 128 x 256 accumulators: while four epilogue warps drain one, the
+// MMA warp fills the other, and the producer and decode warps run straight on into the next tile's stages.
+// Roles (448 threads): warp 0 producer, warp 1 MMA, warps 2..9 decode (two groups, as above), warps 10..13
+// epilogue.  Barriers: the four per-stage barriers of the kernel above, used over one stage sequence that
+// continues across tiles, plus acc_full[2] (tcgen05.commit after a tile's last MMA) and acc_empty[2]
+// (128 epilogue threads after they have read the accumulator).
+constexpr int kPersistThreads = 64 + kDecodeGroups * kDecodeThreads + 128;
+constexpr int kPersistBN = 256;
+
+template <int K>
+__global__ void __launch_bounds__(kPersistThreads, 1)
+gemm_persistent_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
+    constexpr int BN = kPersistBN;
+    using C = Cfg<K, BN>;
+    constexpr int S = C::kStages;
+    extern __shared__ unsigned char smem_raw[];
+    const unsigned base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* smem = smem_raw + (base - smem_u32(smem_raw));
+    const unsigned a_base = base;
+    const unsigned b_base = base + S * kATileBytes;
+    const unsigned p_base = b_base + S * C::kBTileBytes;
+    const unsigned bar_base = p_base + S * C::kPackedBytes;
+    auto full_b = [&](int s) { return bar_base + 8u * s; };
+    auto full_a = [&](int s) { return bar_base + 8u * (S + s); };
+    auto empty = [&](int s) { return bar_base + 8u * (2 * S + s); };
+    auto full_p = [&](int s) { return bar_base + 8u * (3 * S + s); };
+    auto acc_full = [&](int b) { return bar_base + 8u * (4 * S + b); };
+    auto acc_empty = [&](int b) { return bar_base + 8u * (4 * S + 2 + b); };
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(smem + (bar_base - base) + 8 * (4 * S + 4));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nkb = p.in / BK;
+    const int nrt = (p.out + BM - 1) / BM;            // row tiles
+    const int ntt = (p.M + BN - 1) / BN;              // token tiles
+    const int ntiles = nrt * ntt;
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full_b(s), 1);
+            mbar_init(full_a(s), kDecodeThreads);
+            mbar_init(empty(s), 1);
+            mbar_init(full_p(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(acc_full(b), 1);
+            mbar_init(acc_empty(b), 128);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem_d = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- producer ----------------
+        if (lane == 0) {
+            const uint8_t* cbase = p.blob + p.planes_bytes;
+            int it = 0;                                  // stage sequence number, continues across tiles
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+                const int row0 = (tile % nrt) * BM, tok0 = (tile / nrt) * BN;
+                const int nrows = min(BM, p.out - row0);
+                const unsigned seg_p = (unsigned)nrows * 16u, seg_c = (unsigned)nrows * 2u;
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % S;
+                    const unsigned ph = (unsigned)(it / S) & 1u;
+                    if (!mbar_wait(empty(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    const bool first_half = (kb & 1) == 0;
+                    mbar_expect_tx(full_p(s), (first_half ? (unsigned)K * seg_p : 0u) + (unsigned)(K + 1) * seg_c);
+                    const unsigned pdst = p_base + s * C::kPackedBytes;
+                    const int b = kb >> 1, G = (kb * BK) / p.group;
+                    if (first_half) {
+#pragma unroll
+                        for (int i = 0; i < K; ++i)
+                            bulk_load(pdst + i * (BM * 16), p.blob + (((size_t)b * K + i) * p.out + row0) * 16, seg_p, full_p(s));
+                    }
+#pragma unroll
+                    for (int i = 0; i <= K; ++i)
+                        bulk_load(pdst + C::kPlaneBytes + i * (BM * 2), cbase + (((size_t)G * (K + 1) + i) * p.out + row0) * 2, seg_c, full_p(s));
+                    mbar_expect_tx(full_b(s), C::kBTileBytes);
+                    tma_load_2d(b_base + s * C::kBTileBytes, &x_map, kb * BK, tok0, full_b(s));
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            constexpr unsigned idesc = instr_desc_f16(BM, BN);
+            int it = 0, j = 0;                           // stage sequence number; tiles done by this CTA
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++j) {
+                const int buf = j & 1;
+                // the epilogue must have drained this accumulator (two tiles ago)
+                if (!mbar_wait(acc_empty(buf), ((unsigned)(j >> 1) & 1u) ^ 1u, abort_flag, p.status)) break;
+                tc_fence_after();
+                const unsigned d = tmem_d + (unsigned)(buf * BN);
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % S;
+                    const unsigned ph = (unsigned)(it / S) & 1u;
+                    ok = mbar_wait(full_a(s), ph, abort_flag, p.status) && mbar_wait(full_b(s), ph, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t adesc = smem_desc_sw128(a_base + s * kATileBytes);
+                    const uint64_t bdesc = smem_desc_sw128(b_base + s * C::kBTileBytes);
+#pragma unroll
+                    for (int k4 = 0; k4 < BK / 16; ++k4)
+                        umma_f16(d, adesc + 2u * k4, bdesc + 2u * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+                    umma_commit(empty(s));
+                }
+                if (ok) umma_commit(acc_full(buf));
+            }
+        }
+    } else if (warp < 2 + 4 * kDecodeGroups) {
+        // ---------------- decode warps (thread = output row) ----------------
+        const int quad = warp & 3;
+        const int grp = (warp - 2) >> 2;
+        const int rl = quad * 32 + lane;
+        unsigned a_off[8];
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) a_off[ch] = (unsigned)rl * 128u + (((unsigned)ch ^ (unsigned)(rl & 7)) << 4);
+        const int nblocks = nkb / 2;
+        int it0 = 0;                                     // stage sequence number of the current tile's first stage
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, it0 += nkb) {
+            const int r = (tile % nrt) * BM + rl;        // rows past a ragged last tile decode stale bytes; nothing of theirs is stored
+            // A group keeps to every other block of the stage sequence ACROSS tiles (with an odd number of blocks per
+            // tile its parity inside the tile flips): its waits then follow the sequence two stages at a time and
+            // never run a whole ring ahead of a barrier's phase, which a parity wait could not tell from "ready".
+            static_assert(kDecodeGroups == 2, "two groups alternate blocks");
+            for (int b = grp ^ ((it0 >> 1) & 1); b < nblocks && ok; b += kDecodeGroups) {
+                unsigned cur[K][4];
+                bpdq::ByteTables<K> tab;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int it = it0 + 2 * b + half;
+                    const int s = it % S;
+                    const unsigned ph = (unsigned)(it / S) & 1u;
+                    if (!mbar_wait(full_p(s), ph, abort_flag, p.status)) { ok = false; break; }
+                    const unsigned psrc = p_base + s * C::kPackedBytes;
+                    if (half == 0) {
+#pragma unroll
+                        for (int i = 0; i < K; ++i) {
+                            uint4 raw;
+                            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(raw.x), "=r"(raw.y), "=r"(raw.z), "=r"(raw.w)
+                                         : "r"(psrc + i * (BM * 16) + rl * 16));
+                            const uint4 u = bpdq::unrotate_unit(raw, r);
+                            cur[i][0] = u.x; cur[i][1] = u.y; cur[i][2] = u.z; cur[i][3] = u.w;
+                        }
+                    }
+                    if (half == 0 || p.group == 64) {
+                        float c[K + 1];
+#pragma unroll
+                        for (int i = 0; i <= K; ++i) {
+                            unsigned short hbits;
+                            asm volatile("ld.shared.u16 %0, [%1];" : "=h"(hbits) : "r"(psrc + C::kPlaneBytes + i * (BM * 2) + rl * 2));
+                            c[i] = __half2float(__ushort_as_half(hbits));
+                        }
+                        bpdq::candidate_byte_tables<K>(c, tab);
+                    }
+                    const unsigned dst = a_base + s * kATileBytes;
+#pragma unroll
+                    for (int wd = 0; wd < 2; ++wd) {
+                        unsigned w[K], sel[4];
+#pragma unroll
+                        for (int i = 0; i < K; ++i) w[i] = cur[i][2 * half + wd];
+                        bpdq::code_nibbles_word<K>(w, sel);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const uint4 v8 = bpdq::decode8<K>(sel[u], tab);
+                            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + a_off[4 * wd + u]),
+                                         "r"(v8.x), "r"(v8.y), "r"(v8.z), "r"(v8.w) : "memory");
+                        }
+                    }
+                    fence_proxy_async();
+                    mbar_arrive(full_a(s));
+                }
+            }
+        }
+    } else {
+        // ---------------- epilogue warps: drain one accumulator while the other is being filled ----------------
+        const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
+        const int rl = quad * 32 + lane;
+        int j = 0;
+        for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++j) {
+            const int buf = j & 1;
+            if (!mbar_wait(acc_full(buf), (unsigned)(j >> 1) & 1u, abort_flag, p.status)) break;
+            tc_fence_after();
+            const int row0 = (tile % nrt) * BM, tok0 = (tile / nrt) * BN;
+            const int r = row0 + rl;
+            const bool row_ok = r < p.out;
+            const unsigned taddr = tmem_d + ((unsigned)(quad * 32) << 16) + (unsigned)(buf * BN);
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                if (tok0 + c0 >= p.M) break;             // warp-uniform
+                unsigned v[16];
+                tmem_ld16(taddr + (unsigned)c0, v);
+                tmem_ld_wait();
+                if (row_ok) {
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj) {
+                        const int t = tok0 + c0 + jj;
+                        if (t < p.M) p.y[(size_t)t * p.out + r] = __float2half_rn(__uint_as_float(v[jj]));
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty(buf));                 // 128 arrivals: the accumulator may be overwritten
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_d, 512);
+    }
+}
+
 // ---- host side ------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -438,11 +668,44 @@ int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t st
 }
 
 template <int K>
+int launch_persistent(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
+    using C = Cfg<K, kPersistBN>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_persistent_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: shared memory opt-in: %s", cudaGetErrorString(e));
+        configured = true;
+    }
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: cuTensorMapEncodeTiled is not available from this driver");
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)h->in, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)h->in * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)kPersistBN};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult cr = enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: tensor map encode failed (CUresult %d)", (int)cr);
+    GemmParams p;
+    p.blob = h->d_blob; p.planes_bytes = h->planes_bytes; p.y = static_cast<__half*>(y); p.status = h->d_status;
+    p.out = h->out; p.in = h->in; p.group = h->group; p.M = M;
+    p.ws = h->d_ws; p.counters = h->d_counters; p.kb_per = h->in / BK;
+    const long long ntiles = (long long)((h->out + BM - 1) / BM) * ((M + kPersistBN - 1) / kPersistBN);
+    const int grid = ntiles < h->sm_count ? (int)ntiles : h->sm_count;
+    gemm_persistent_kernel<K><<<grid, kPersistThreads, C::kSmemBytes, stream>>>(map, p);
+    h->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm launch: %s", cudaGetErrorString(e));
+    return BPDQ_OK;
+}
+
+template <int K>
 int launch_k(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
     if (M <= 32) return launch_tile<K, 32>(h, x, y, M, stream);
     if (M <= 64) return launch_tile<K, 64>(h, x, y, M, stream);
     if (M <= 128) return launch_tile<K, 128>(h, x, y, M, stream);
-    return launch_tile<K, 256>(h, x, y, M, stream);
+    return launch_persistent<K>(h, x, y, M, stream);
 }
 
 }  // namespace

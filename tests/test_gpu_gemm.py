@@ -25,11 +25,16 @@ pytestmark = pytest.mark.gpu
     (2, 128, 256, 4096, 40),     # few row tiles, long rows: four CTAs share an output tile (split over the input dimension)
     (3, 64, 128, 8192, 64),      # eight-way split
     (4, 128, 384, 2048, 7),      # two-way split, ragged token tile
+    (2, 128, 256, 384, 20500),   # 162 output tiles for 148 persistent CTAs: a second tile per CTA, odd number of blocks per tile
+    (4, 128, 128, 640, 38000),   # 149 tiles, three-stage ring (K = 4), odd number of blocks per tile
 ])
 def test_gemm_kernel(K, g, out, in_, M):
     h, bits, coef = G.make_layer(60 + K, out, in_, K, g, max_M=M)
     x = synth.activations(70 + K, M, in_)
-    G.check_linear(h, bits, coef, x, g, binding.KERNEL_GEMM, what="gemm")
+    rows = None
+    if M > 4096:                 # many tokens: every token, rows sampled from every 32-row quadrant of every row tile
+        rows = np.unique(np.concatenate([np.arange(0, out, 37), [0, 31, 32, 127, out - 128, out - 1]]))
+    G.check_linear(h, bits, coef, x, g, binding.KERNEL_GEMM, rows=rows, what="gemm")
     y1 = G.run_linear(h, x, binding.KERNEL_GEMM)
     y2 = G.run_linear(h, x, binding.KERNEL_GEMM)
     if M > 64 or in_ < 2048:
