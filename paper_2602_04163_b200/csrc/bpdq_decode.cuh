@@ -40,19 +40,35 @@ __device__ __forceinline__ unsigned code_nibbles(const unsigned (&w)[K], const i
 // Codes of all 32 columns of one logical word: sel[u] holds, in nibble j, the code of column 8u + j.
 template <int K>
 __device__ __forceinline__ void code_nibbles_word(const unsigned (&w)[K], unsigned (&sel)[4]) {
-    if constexpr (K == 2) {
-        // interleave the two planes once: e has plane 0 on even and plane 1 on odd bit positions
-        // for the columns at even positions of the word, o the same for the odd positions
-        const unsigned m = 0x55555555u;
-        const unsigned e = (w[0] & m) | ((w[1] << 1) & ~m);
-        const unsigned o = ((w[0] >> 1) & m) | (w[1] & ~m);
-        sel[0] = e & 0x33333333u;
-        sel[1] = o & 0x33333333u;
-        sel[2] = (e >> 2) & 0x33333333u;
-        sel[3] = (o >> 2) & 0x33333333u;
-    } else {
+    // Interleave planes 0 and 1 once: e has plane 0 on even and plane 1 on odd bit positions for the columns at
+    // even positions of the word (u = 0, 2), o the same for the odd positions (u = 1, 3); two-bit codes then
+    // come out with one mask.  Planes 2 and 3 are interleaved the same way and land two bits higher.
+    const unsigned m5 = 0x55555555u, m3 = 0x33333333u;
+    if constexpr (K == 1) {
 #pragma unroll
         for (int u = 0; u < 4; ++u) sel[u] = code_nibbles<K>(w, u);
+    } else {
+        const unsigned e = (w[0] & m5) | ((w[1] << 1) & ~m5);
+        const unsigned o = ((w[0] >> 1) & m5) | (w[1] & ~m5);
+        if constexpr (K == 2) {
+            sel[0] = e & m3;
+            sel[1] = o & m3;
+            sel[2] = (e >> 2) & m3;
+            sel[3] = (o >> 2) & m3;
+        } else if constexpr (K == 3) {
+            const unsigned m4 = 0x44444444u;          // plane 2 goes to bit 2 of every nibble
+            sel[0] = (e & m3) | ((w[2] << 2) & m4);
+            sel[1] = (o & m3) | ((w[2] << 1) & m4);
+            sel[2] = ((e >> 2) & m3) | (w[2] & m4);
+            sel[3] = ((o >> 2) & m3) | ((w[2] >> 1) & m4);
+        } else {
+            const unsigned e2 = (w[2] & m5) | ((w[3] << 1) & ~m5);
+            const unsigned o2 = ((w[2] >> 1) & m5) | (w[3] & ~m5);
+            sel[0] = (e & m3) | ((e2 << 2) & ~m3);
+            sel[1] = (o & m3) | ((o2 << 2) & ~m3);
+            sel[2] = ((e >> 2) & m3) | (e2 & ~m3);
+            sel[3] = ((o >> 2) & m3) | (o2 & ~m3);
+        }
     }
 }
 
