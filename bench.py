@@ -447,6 +447,29 @@ def extra_sections(torch, binding, args, peaks, sp, stream):
             for h in L:
                 h.bpdq_destroy()
 
+    # Qwen2.5-7B-shaped layer (69 MB packed at K = 2: five copies rotated to stay out of L2), one batched launch
+    for K in (2, 3):
+        shapes7b = synth.QWEN25_7B_LAYER
+        copies = 5
+        layers = [[binding.Handle(o, i, K, GROUP, None, 900 + 10 * c + li, 1) for li, (_, o, i) in enumerate(shapes7b)] for c in range(copies)]
+        xs = {i: xt(1, i) for i in sorted({i for _, _, i in shapes7b})}
+        ys = [torch.empty((1, o), dtype=torch.float16, device="cuda") for _, o, _ in shapes7b]
+        b = layer_bytes(shapes7b, K, 1)
+        n = 100
+
+        def run_7b():
+            for k in range(n):
+                hs = layers[k % copies]
+                binding.bpdq_linear_batch(hs, [xs[h.in_].data_ptr() for h in hs], [y.data_ptr() for y in ys], 1, sp)
+        run_7b()
+        ms = event_time_ms(torch, run_7b, stream) / n
+        out[f"gemv_layer_7b_batched_K{K}"] = {"launches_per_layer": 1, "us_per_layer": ms * 1e3, "gbs": b / (ms * 1e-3) / 1e9,
+                                              "frac_measured": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                              "l2": f"{copies} layer copies of {b / 1e6:.0f} MB rotated"}
+        for L in layers:
+            for h in L:
+                h.bpdq_destroy()
+
     # token-count sweep on the gate and down projections: both kernels, to place the dispatch threshold
     sweep = []
     for K in (2, 3):
