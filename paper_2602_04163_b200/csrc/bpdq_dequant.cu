@@ -1,12 +1,14 @@
 // bpdq_dequant: materialise W^ (Eq. 1) as binary16 [out][in].
 //
 // One warp owns 32 rows x one 128-column block.  Lane l reads its row's K plane units
-// (consecutive rows are adjacent in the blob: one coalesced 512-byte request per plane) and
-// builds the 2^K candidate values of its (row, group) (Eq. 7) with the decode rule's exact
-// arithmetic: float(c0), then "+ float(ci)" in binary32 for the set bits in plane order, one
-// rounding to binary16.  Units and candidate tables are staged in shared memory; the warp then
-// writes two rows per step, 16 lanes x 16 bytes each (eight consecutive columns: one bit per nibble of a logical word), so every row segment leaves as one
-// contiguous 256-byte store.  HBM-bound on the 2 bytes per weight it writes.
+// (consecutive rows are adjacent in the blob: one coalesced 512-byte request per plane), undoes the
+// row's byte rotation, and builds the 2^K candidate values of its (row, group) (Eq. 7) with the
+// decode rule's exact arithmetic: float(c0), then "+ float(ci)" in binary32 for the set bits in
+// plane order, one rounding to binary16 -- kept as byte tables for the byte-permute decode that
+// the tensor-core kernel uses too.  Units and tables are staged in shared memory; the warp then
+// writes two rows per step, 16 lanes x 16 bytes each (eight consecutive columns: one bit per
+// nibble of a logical word, turned into eight binary16 by eight byte-permutes), so every row
+// segment leaves as one contiguous 256-byte store.  HBM-bound on the 2 bytes per weight it writes.
 #include "bpdq_internal.h"
 #include "bpdq_decode.cuh"
 
@@ -20,9 +22,9 @@ template <int K>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 dequant_kernel(const uint8_t* __restrict__ blob, size_t planes_bytes, __half* __restrict__ w, int out, int in,
                int group) {
-    constexpr int NC = 1 << K;                       // candidate values per group
-    __shared__ __align__(16) uint8_t s_units[kWarpsPerCta][K][32][16];
-    __shared__ __align__(16) __half s_table[kWarpsPerCta][32][2][NC];
+    constexpr int NT = K == 4 ? 4 : 2;               // table words per half (low bytes, high bytes)
+    __shared__ __align__(16) unsigned s_units[kWarpsPerCta][32][K][4];          // logical words, per row
+    __shared__ __align__(16) unsigned s_tab[kWarpsPerCta][32][2][2 * NT];       // per row and 64-column half: lo[NT], hi[NT]
 
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int nblocks = in / 128;
@@ -40,7 +42,7 @@ dequant_kernel(const uint8_t* __restrict__ blob, size_t planes_bytes, __half* __
 #pragma unroll
             for (int i = 0; i < K; ++i) {
                 const uint4 u = *reinterpret_cast<const uint4*>(blob + bpdq::plane_unit_offset(b, i, r, K, out));
-                *reinterpret_cast<uint4*>(&s_units[wid][i][lane][0]) = bpdq::unrotate_unit(u, r);   // staged in logical byte order
+                *reinterpret_cast<uint4*>(&s_units[wid][lane][i][0]) = bpdq::unrotate_unit(u, r);   // staged in logical byte order
             }
             for (int sub = 0; sub < nsub; ++sub) {
                 const int G = (b * 128 + sub * 64) / group;
@@ -48,39 +50,34 @@ dequant_kernel(const uint8_t* __restrict__ blob, size_t planes_bytes, __half* __
 #pragma unroll
                 for (int i = 0; i <= K; ++i)
                     c[i] = __half2float(*reinterpret_cast<const __half*>(cbase + bpdq::coef_offset(G, i, r, K, out)));
+                bpdq::ByteTables<K> t;
+                bpdq::candidate_byte_tables<K>(c, t);
 #pragma unroll
-                for (int code = 0; code < NC; ++code) {
-                    float acc = c[0];
-#pragma unroll
-                    for (int i = 0; i < K; ++i)
-                        if ((code >> i) & 1) acc = __fadd_rn(acc, c[i + 1]);
-                    s_table[wid][lane][sub][code] = __float2half_rn(acc);
+                for (int k = 0; k < NT; ++k) {
+                    s_tab[wid][lane][sub][k] = t.lo[k];
+                    s_tab[wid][lane][sub][NT + k] = t.hi[k];
                 }
             }
         }
         __syncwarp();
-        const int c8 = lane & 15;                    // logical 8-column chunk this lane writes
+        const int c8 = lane & 15;                    // eight-column chunk this lane writes: word c8 / 4, phase u = c8 % 4
         const int sub = (group == 64) ? (c8 >> 3) : 0;
 #pragma unroll 4
         for (int it = 0; it < 16; ++it) {
             const int lr = it * 2 + (lane >> 4);     // local row
             const int rr = rb * 32 + lr;
             if (rr < out) {
-                // columns 8*c8 .. 8*c8+7 are bits 4*t + u of logical word k, k = c8 / 4, u = c8 % 4
                 unsigned word[K];
 #pragma unroll
-                for (int i = 0; i < K; ++i)
-                    word[i] = *reinterpret_cast<const unsigned*>(&s_units[wid][i][lr][(c8 >> 2) * 4]) >> (c8 & 3);
-                __align__(16) __half v[8];
+                for (int i = 0; i < K; ++i) word[i] = s_units[wid][lr][i][c8 >> 2];
+                bpdq::ByteTables<K> t;
 #pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    unsigned code = 0;
-#pragma unroll
-                    for (int i = 0; i < K; ++i) code |= ((word[i] >> (4 * t)) & 1u) << i;
-                    v[t] = s_table[wid][lr][sub][code];
+                for (int k = 0; k < NT; ++k) {
+                    t.lo[k] = s_tab[wid][lr][sub][k];
+                    t.hi[k] = s_tab[wid][lr][sub][NT + k];
                 }
-                *reinterpret_cast<uint4*>(w + (size_t)rr * in + (size_t)b * 128 + c8 * 8) =
-                    *reinterpret_cast<const uint4*>(v);
+                const uint4 v = bpdq::decode8<K>(bpdq::code_nibbles<K>(word, c8 & 3), t);
+                *reinterpret_cast<uint4*>(w + (size_t)rr * in + (size_t)b * 128 + c8 * 8) = v;
             }
         }
         __syncwarp();
