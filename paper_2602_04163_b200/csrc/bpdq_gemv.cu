@@ -174,6 +174,70 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
     const int t_end = p.t_begin[bid + 1];
     int li = 0;                                       // linear that task t belongs to
 
+    // ---- hand-over of a finished segment ----
+    // Row sums are accumulated across slices with binary32 atomic adds in `ws` (kept zero
+    // between calls).  Row groups are counted in chunks of kChunkRgs; whoever delivers the last
+    // contribution of a chunk converts its rows to binary16, writes y and zeroes `ws` again.
+    // The caller has fenced the segment's atomic adds and passed a CTA barrier.
+    auto hand_over = [&](const GemvLinear& L, const int rg_begin, const int rg_end) {
+        const int ck_begin = rg_begin / kChunkRgs, ck_end = (rg_end + kChunkRgs - 1) / kChunkRgs;
+        for (int ck0 = ck_begin; ck0 < ck_end; ck0 += kMaxDone) {
+            if (tid == 0) *ndone = 0;
+            __syncthreads();
+            for (int ck = ck0 + tid; ck < min(ck_end, ck0 + kMaxDone); ck += kThreads) {
+                const int lo = max(rg_begin, ck * kChunkRgs), hi = min(rg_end, (ck + 1) * kChunkRgs);
+                const int size = min(L.nrg, (ck + 1) * kChunkRgs) - ck * kChunkRgs;
+                const unsigned before = atomicAdd(&L.counters[ck], (unsigned)(hi - lo));
+                if (before + (unsigned)(hi - lo) == (unsigned)(size * L.nslices)) {
+                    L.counters[ck] = 0u;
+                    done[atomicAdd(ndone, 1)] = ck;
+                }
+            }
+            __syncthreads();
+            const int nd = *ndone;
+            if (nd > 0) {
+                __threadfence();
+                // items of four consecutive rows; a thread reads several before it writes, so that the
+                // L2 round trips of a CTA that completes many chunks overlap
+                constexpr int kQuads = kChunkRgs * 16 / 4, kAhead = 4;
+                const int nitems = nd * MT * kQuads;
+                for (int i0 = tid; i0 < nitems; i0 += kThreads * kAhead) {
+                    float4 v[kAhead];
+                    size_t at[kAhead];
+                    bool live[kAhead];
+#pragma unroll
+                    for (int u = 0; u < kAhead; ++u) {
+                        const int idx = i0 + u * kThreads;
+                        live[u] = false;
+                        if (idx < nitems) {
+                            const int ckd = done[idx / (MT * kQuads)];
+                            const int rem = idx % (MT * kQuads);
+                            const int r = ckd * kChunkRgs * 16 + (rem % kQuads) * 4;
+                            if (r < L.out) {                  // out is a multiple of 16: a quad is inside or outside as a whole
+                                live[u] = true;
+                                at[u] = (size_t)(rem / kQuads) * L.out + r;
+                                v[u] = __ldcg(reinterpret_cast<const float4*>(L.ws + at[u]));
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < kAhead; ++u) {
+                        if (live[u]) {
+                            const __half2 h01 = __floats2half2_rn(v[u].x, v[u].y), h23 = __floats2half2_rn(v[u].z, v[u].w);
+                            uint2 o;
+                            o.x = *reinterpret_cast<const unsigned*>(&h01);
+                            o.y = *reinterpret_cast<const unsigned*>(&h23);
+                            *reinterpret_cast<uint2*>(L.y + at[u]) = o;
+                            __stcg(reinterpret_cast<float4*>(L.ws + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    };
+    int pend_li = -1, pend_begin = 0, pend_end = 0;   // finished segment whose hand-over is still due
+
     while (t < t_end) {
         while (li + 1 < p.n && t >= p.lin[li + 1].task_begin) ++li;
         const GemvLinear& L = p.lin[li];
@@ -258,6 +322,9 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
             for (int d = 0; d < D; ++d)
                 if (d < ntask) load_task(tk[d], d);
         }
+
+        // the previous segment is handed over while this segment's first loads are in flight
+        if (pend_li >= 0) hand_over(p.lin[pend_li], pend_begin, pend_end);
 
         // ---- build the 64 chunk tables of this slice (per token) ----
 #pragma unroll
@@ -421,45 +488,13 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
             }
         }
 
-        // ---- hand this segment over ----
-        // Row sums are accumulated across slices with binary32 atomic adds in `ws` (kept zero
-        // between calls).  Row groups are counted in chunks of kChunkRgs; whoever delivers the last
-        // contribution of a chunk converts its rows to binary16, writes y and zeroes `ws` again.
+        // ---- segment finished: its atomic adds are fenced, all warps are done with the tables ----
         __threadfence();
         __syncthreads();
-        const int ck_begin = rg_begin / kChunkRgs, ck_end = (rg_end + kChunkRgs - 1) / kChunkRgs;
-        for (int ck0 = ck_begin; ck0 < ck_end; ck0 += kMaxDone) {
-            if (tid == 0) *ndone = 0;
-            __syncthreads();
-            for (int ck = ck0 + tid; ck < min(ck_end, ck0 + kMaxDone); ck += kThreads) {
-                const int lo = max(rg_begin, ck * kChunkRgs), hi = min(rg_end, (ck + 1) * kChunkRgs);
-                const int size = min(L.nrg, (ck + 1) * kChunkRgs) - ck * kChunkRgs;
-                const unsigned before = atomicAdd(&L.counters[ck], (unsigned)(hi - lo));
-                if (before + (unsigned)(hi - lo) == (unsigned)(size * L.nslices)) {
-                    L.counters[ck] = 0u;
-                    done[atomicAdd(ndone, 1)] = ck;
-                }
-            }
-            __syncthreads();
-            const int nd = *ndone;
-            if (nd > 0) {
-                __threadfence();
-                for (int idx = tid; idx < nd * kChunkRgs * 16 * MT; idx += kThreads) {
-                    const int ckd = done[idx / (kChunkRgs * 16 * MT)];
-                    const int rem = idx % (kChunkRgs * 16 * MT);
-                    const int m = rem / (kChunkRgs * 16);
-                    const int r = ckd * kChunkRgs * 16 + rem % (kChunkRgs * 16);
-                    if (r < L.out) {
-                        float* src = L.ws + (size_t)m * L.out + r;
-                        L.y[(size_t)m * L.out + r] = __float2half_rn(__ldcg(src));
-                        __stcg(src, 0.f);
-                    }
-                }
-            }
-            __syncthreads();
-        }
+        pend_li = li; pend_begin = rg_begin; pend_end = rg_end;
         t += rg_end - rg_begin;
     }
+    if (pend_li >= 0) hand_over(p.lin[pend_li], pend_begin, pend_end);
 }
 
 template <int K, int MT, int D, int W, bool G64>
