@@ -102,6 +102,13 @@ __device__ __forceinline__ float lds_table(unsigned addr) {
     asm("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"(IMM));
     return v;
 }
+// prmt.b32 in its generic form: selector nibble n picks byte n of {b, a} (a = bytes 0..3); with its top bit set
+// the byte's sign is replicated instead
+__device__ __forceinline__ unsigned prmt(unsigned a, unsigned b, unsigned sel) {
+    unsigned d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
 __device__ __forceinline__ unsigned word_of(const uint4& v, int k) {
     return k == 0 ? v.x : k == 1 ? v.y : k == 2 ? v.z : v.w;
 }
@@ -156,13 +163,23 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
     int* ndone = done + kMaxDone;
     float* lut = reinterpret_cast<float*>(smem + (lut0 - smem0));         // [MT][256][kSlots]
 
-    // the lane's table-slot address per step: lut0 + 4*((s + a) mod 16) + 64*h; the plane byte is
-    // spliced into bits 8..15 (entry row stride 256 B)
-    unsigned off[16];
+    // The lane's table address at step s is lut0 + 256 * (plane byte) + slot(s), slot(s) = 4*((s + a) mod 16) + 64*h
+    // (< 128).  lut0 is a multiple of 64 KB below 16 MB, so the address is four bytes: [slot][plane byte]
+    // [lut0 >> 16][0], which one byte-permute assembles from the plane word and a register that holds
+    // lut0 >> 16 in byte 0 and the slots of three consecutive steps in bytes 1..3 (the zero top byte is
+    // the replicated sign of byte 0).
+    unsigned slots[6];
 #pragma unroll
-    for (int s = 0; s < 16; ++s) off[s] = lut0 + 4u * ((s + a) & 15) + 64u * h;
+    for (int j = 0; j < 6; ++j) {
+        slots[j] = lut0 >> 16;
 #pragma unroll
-    for (int s = 0; s < 16; ++s) asm volatile("" : "+r"(off[s]));   // opaque: kept in registers instead of being recomputed at every use
+        for (int e = 0; e < 3; ++e) {
+            const int s = 3 * j + e;
+            if (s < 16) slots[j] |= (4u * ((s + a) & 15) + 64u * h) << (8 * (e + 1));
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 6; ++j) asm volatile("" : "+r"(slots[j]));   // opaque: kept in registers instead of being recomputed at every use
     // steps at which this lane's chunk (logical byte (s + a) mod 16) lies in the block's first 64 columns
     unsigned lo_steps = 0;
 #pragma unroll
@@ -385,7 +402,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                     unsigned addr[K];
 #pragma unroll
                     for (int i = 0; i < K; ++i)
-                        addr[i] = __byte_perm(word_of(tk.pl[q][i], st >> 2), off[st], 0x7604u | ((st & 3) << 4));
+                        addr[i] = prmt(word_of(tk.pl[q][i], st >> 2), slots[st / 3], 0xC400u | ((st & 3) << 4) | (5 + st % 3));   // the selector is a constant once the step loop is unrolled
                     constexpr int QI = 128;               // the block pair and the token's table go into the immediate
                     if constexpr (G64) {
                         float v[NS];
@@ -514,57 +531,56 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
         total += (long long)p.lin[k].nslices * p.lin[k].nrg;
         if (total >= (1ll << 31)) return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv: task space too large");
     }
-    // Cut the task space into one share per SM of equal cost, a segment (a CTA's visit to one slice
-    // of one linear: table set-up, hand-over) counting as kSegmentCost tasks.  Short slices (few
-    // output rows) would otherwise load the CTAs that get them with many set-ups.
+    // Cut the task space into one contiguous share per SM such that the most expensive share is as
+    // cheap as possible, a segment (a CTA's visit to one slice of one linear: table set-up, drain,
+    // hand-over) counting as kSegmentCost tasks.  Short slices (few output rows) would otherwise load
+    // the CTAs that get them with many set-ups.  The smallest feasible bound is found by bisection: for
+    // a given bound every CTA in turn takes as many tasks as fit under it.
     int grid = h->sm_count < kMaxGrid ? h->sm_count : kMaxGrid;
     if ((long long)grid > total) grid = (int)total;
-    {
-        const int kSegmentCost = p.n > 1 ? kSegmentCostBatch : kSegmentCostSingle;
-        long long nseg = 0;
-        for (int k = 0; k < p.n; ++k) nseg += p.lin[k].nslices;
-        // cost of the tasks [t0, t1) as one CTA's share
-        auto share_cost = [&](long long t0, long long t1) {
-            long long cost = 0;
-            int k = 0;
-            for (long long t = t0; t < t1;) {
-                while (k + 1 < p.n && t >= p.lin[k + 1].task_begin) ++k;
-                const long long in_slice = p.lin[k].nrg - (t - p.lin[k].task_begin) % p.lin[k].nrg;
-                const long long take = in_slice < t1 - t ? in_slice : t1 - t;
-                cost += kSegmentCost + take;
-                t += take;
-            }
-            return cost;
-        };
-        double target = (double)(total + nseg * kSegmentCost) / grid;
-        for (int round = 0; round < 8; ++round) {     // cuts inside slices add segments: raise the target until the last share fits
-            int b = 0, k = 0;
-            long long t = 0;                          // next unassigned task
+    const int kSegmentCost = p.n > 1 ? kSegmentCostBatch : kSegmentCostSingle;
+    static_assert(sizeof(h->plan_t_begin) == sizeof(p.t_begin), "one cached entry per CTA boundary");
+    bool cached = h->plan_n == p.n && h->plan_cost == kSegmentCost && h->plan_grid == grid;
+    for (int k = 0; cached && k < p.n; ++k) cached = h->plan_shape[k][0] == p.lin[k].nrg && h->plan_shape[k][1] == p.lin[k].nslices;
+    if (cached) {
+        for (int c = 0; c <= grid; ++c) p.t_begin[c] = h->plan_t_begin[c];
+    } else {
+        constexpr int kMinSegment = 8;                // a share is closed rather than opened into a slice for fewer tasks than this
+        // fills t_begin for the bound; true when `grid` shares cover the task space
+        auto sweep = [&](const double bound) {
+            long long t = 0;
+            int k = 0, b = 0;
             p.t_begin[0] = 0;
-            double budget = target;
-            while (t < total && b < grid - 1) {
-                while (k + 1 < p.n && t >= p.lin[k + 1].task_begin) ++k;
-                const long long in_slice = p.lin[k].nrg - (t - p.lin[k].task_begin) % p.lin[k].nrg;   // tasks left in the current slice
-                if (budget < kSegmentCost + 8 && t > p.t_begin[b]) {         // not worth opening another segment here
-                    p.t_begin[++b] = (int)t;
-                    budget += target;
-                    continue;
+            while (t < total && b < grid) {
+                double budget = bound;
+                const long long start = t;
+                while (t < total) {
+                    while (k + 1 < p.n && t >= p.lin[k + 1].task_begin) ++k;
+                    const long long in_slice = p.lin[k].nrg - (t - p.lin[k].task_begin) % p.lin[k].nrg;   // tasks left in the current slice
+                    const double room = budget - kSegmentCost;
+                    if (t > start && room < (double)(in_slice < kMinSegment ? in_slice : kMinSegment)) break;
+                    long long take = room >= 1.0 ? (long long)room : 1;
+                    if (take > in_slice) take = in_slice;
+                    t += take;
+                    budget -= (double)(kSegmentCost + take);
+                    if (take < in_slice) break;
                 }
-                budget -= kSegmentCost;
-                long long take = in_slice;
-                if ((double)take > budget) take = (long long)budget > 0 ? (long long)budget : 1;
-                t += take;
-                budget -= (double)take;
-                if (take < in_slice) {                                        // budget spent inside the slice
-                    p.t_begin[++b] = (int)t;
-                    budget += target;
-                }
+                p.t_begin[++b] = (int)t;
             }
-            for (int c = b + 1; c <= grid; ++c) p.t_begin[c] = (int)total;    // the last share takes what is left
-            const double last = (double)share_cost(p.t_begin[b], total);
-            if (last <= 1.05 * target) break;
-            target += (last - target) / grid;
+            const bool covered = t >= total;
+            for (int c = b + 1; c <= grid; ++c) p.t_begin[c] = (int)total;
+            return covered;
+        };
+        double lo = (double)total / grid, hi = 2.0 * (double)total / grid + 16.0 * kSegmentCost + 16.0;
+        while (!sweep(hi)) hi *= 2.0;                 // terminates: a bound above the whole cost covers everything
+        for (int it = 0; it < 24 && hi - lo > 0.5; ++it) {
+            const double mid = 0.5 * (lo + hi);
+            if (sweep(mid)) hi = mid; else lo = mid;
         }
+        sweep(hi);
+        h->plan_n = p.n; h->plan_cost = kSegmentCost; h->plan_grid = grid;
+        for (int k = 0; k < p.n; ++k) { h->plan_shape[k][0] = p.lin[k].nrg; h->plan_shape[k][1] = p.lin[k].nslices; }
+        for (int c = 0; c <= grid; ++c) h->plan_t_begin[c] = p.t_begin[c];
     }
     p.dyn_smem = smem;
     cudaLaunchConfig_t cfg = {};

@@ -51,6 +51,11 @@ struct bpdq_handle_s {
     void* d_ystage;
     int gemv_max_m;
     uint64_t launches;
+    // Last cut of a look-up-table launch led by this handle (the cut depends on the shapes only): linears,
+    // their (row groups, slices), segment cost, CTAs, first task of every CTA.  plan_n == 0: none yet.
+    int plan_n, plan_cost, plan_grid;
+    int plan_shape[BPDQ_BATCH_MAX][2];
+    int plan_t_begin[193];
 };
 
 // Kernel launchers (each returns a BPDQ_* status; all asynchronous on `stream`).
