@@ -45,7 +45,7 @@ constexpr int kMaxDone = 512;                         // completed chunks handle
 // (slice, row group) task spaces are concatenated and every CTA takes a contiguous share of the whole.
 struct GemvLinear {
     const uint8_t* blob;
-    size_t planes_bytes;
+    size_t planes_bytes, blob_bytes;
     const __half* x;          // [MT][in]
     __half* y;                // [MT][out]
     float* ws;                // [MT][out] binary32 row sums, zero between calls
@@ -258,9 +258,10 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
     while (t < t_end) {
         while (li + 1 < p.n && t >= p.lin[li + 1].task_begin) ++li;
         const GemvLinear& L = p.lin[li];
-        const uint8_t* cbase = L.blob + L.planes_bytes;
-        const size_t plane_pitch = (size_t)L.out * 16;    // bytes between planes of one block
-        const size_t coef_pitch = (size_t)L.out * 2;      // bytes between coefficients of one group
+        // byte offsets into the blob fit 32 bits (the launcher refuses larger blobs): addresses are the blob's
+        // uniform base plus a 32-bit per-lane offset
+        const unsigned plane_pitch = (unsigned)L.out * 16u;   // bytes between planes of one block
+        const unsigned coef_pitch = (unsigned)L.out * 2u;     // bytes between coefficients of one group
         const int tl = t - L.task_begin;
         const int s = tl / L.nrg;
         const int rg_begin = tl - s * L.nrg;
@@ -268,8 +269,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
         const int ntask = (rg_end - rg_begin - wid + W - 1) / W;          // tasks of this warp (may be <= 0)
 
         // per-lane source pointers of the first task; a task further on is W*16 rows further on
-        const uint8_t* psrc[2];
-        const uint8_t* csrc[2];
+        unsigned psrc[2], csrc[2];
         bool valid[2];
         {
             const int r = (rg_begin + wid) * 16 + a;
@@ -278,23 +278,23 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                 const int b = s * kSliceBlocks + 2 * q + h;
                 valid[q] = b < L.nblocks;                                  // false past the end of a ragged last slice
                 const int bb = valid[q] ? b : 0;
-                psrc[q] = L.blob + ((size_t)bb * K * L.out + r) * 16;
+                psrc[q] = ((unsigned)bb * K * L.out + r) * 16u;
                 const int G = (bb * 128) / L.group;
-                csrc[q] = cbase + ((size_t)G * (K + 1) * L.out + r) * 2;
+                csrc[q] = (unsigned)L.planes_bytes + ((unsigned)G * (K + 1) * L.out + r) * 2u;
             }
         }
         auto load_task = [&](Task<K, NG>& tk, int n) {
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 if (valid[q]) {
-                    const uint8_t* ps = psrc[q] + (size_t)n * (W * 256);
+                    const unsigned ps = psrc[q] + (unsigned)n * (W * 256);
 #pragma unroll
-                    for (int i = 0; i < K; ++i) tk.pl[q][i] = ldg_stream16(ps + i * plane_pitch);
-                    const uint8_t* cs = csrc[q] + (size_t)n * (W * 32);
+                    for (int i = 0; i < K; ++i) tk.pl[q][i] = ldg_stream16(L.blob + (size_t)(ps + i * plane_pitch));
+                    const unsigned cs = csrc[q] + (unsigned)n * (W * 32);
 #pragma unroll
                     for (int gg = 0; gg < NG; ++gg)
 #pragma unroll
-                        for (int i = 0; i <= K; ++i) tk.cf[q][gg][i] = ldg_stream2(cs + (gg * (K + 1) + i) * coef_pitch);
+                        for (int i = 0; i <= K; ++i) tk.cf[q][gg][i] = ldg_stream2(L.blob + (size_t)(cs + (gg * (K + 1) + i) * coef_pitch));
                 } else {                              // contributes nothing: zero planes, zero coefficients
 #pragma unroll
                     for (int i = 0; i < K; ++i) tk.pl[q][i] = make_uint4(0u, 0u, 0u, 0u);
@@ -527,6 +527,8 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     }
     long long total = 0;
     for (int k = 0; k < p.n; ++k) {
+        if ((unsigned long long)p.lin[k].blob_bytes >= (1ull << 32))
+            return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv: packed weights of 4 GB or more in one linear");
         p.lin[k].task_begin = (int)total;
         total += (long long)p.lin[k].nslices * p.lin[k].nrg;
         if (total >= (1ll << 31)) return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv: task space too large");
@@ -596,17 +598,19 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     return BPDQ_OK;
 }
 
-// Tasks kept in flight per lane: two (a third costs more in recomputed addresses than it hides in latency);
-// one when the second coefficient group of g = 64 takes the registers (K >= 3).
+// Tasks kept in flight per lane: two (a third costs more in registers than it hides in latency: measured slower
+// for every K); one where two tasks do not fit the register file (K = 4; K >= 3 with the second coefficient
+// group of g = 64).
 template <int K, int MT>
 int launch_one(bpdq_handle_s* h, const GemvParams& p, cudaStream_t stream) {
     if (p.lin[0].group == 64) return launch_cfg<K, MT, (K <= 2 ? 2 : 1), 16, true>(h, p, stream);
-    return launch_cfg<K, MT, 2, 16, false>(h, p, stream);
+    return launch_cfg<K, MT, (K <= 3 ? 2 : 1), 16, false>(h, p, stream);
 }
 
 void fill_linear(GemvLinear& L, const bpdq_handle_s* h) {
     L.blob = h->d_blob;
     L.planes_bytes = h->planes_bytes;
+    L.blob_bytes = h->blob_bytes;
     L.ws = h->d_ws;
     L.counters = h->d_counters;
     L.out = h->out; L.in = h->in; L.group = h->group;
