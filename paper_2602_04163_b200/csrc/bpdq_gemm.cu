@@ -12,13 +12,16 @@
 // 16-byte chunk c of row r is stored at chunk position c ^ (r mod 8).  TMA writes that layout by
 // itself; the decode threads reproduce it by hand.
 //
-// Roles (320 threads): warp 0 issues the TMA loads of x; warp 1 allocates TMEM and issues the
-// MMAs (one lane); warps 2..9 decode in two groups of four warps, thread = output row, group 0
-// taking the even 128-column blocks (two stages each) and group 1 the odd ones (one warp per
-// scheduler could not hide its own instruction latencies).  The packed planes and coefficients of a stage come
-// through the same pipeline as x: for every stage the producer also issues bulk copies of the K
-// plane segments (128 rows x 16 bytes, contiguous in the blob; once per 128-column block, with
-// the block's first stage) and the K+1 coefficient segments (128 rows x 2 bytes) of the tile's rows, so that no decode thread ever waits on global memory.
+// Roles (320 threads): warp 0 is the producer (one lane: TMA loads of x and of the packed weights);
+// warp 1 allocates TMEM and issues the MMAs (one lane); warps 2..9 decode in two groups of four
+// warps, thread = output row, group 0 taking the even 128-column blocks (two stages each) and
+// group 1 the odd ones (one warp per scheduler could not hide its own instruction latencies).
+// The packed planes and coefficients come through the pipeline as well, so that no decode thread
+// ever waits on global memory: in the tile kernel a block's K plane segments (128 rows x 16 bytes)
+// are one box of a tensor map over the blob's planes and its coefficient segments (128 rows x
+// 2 bytes) one box of a map over the coefficients -- two copies per block whatever K is (the TMA
+// unit takes about 55 ns per copy however small, and 2K+1 bulk copies per block made the kernel
+// slower with every plane); the persistent kernel issues bulk copies per segment.
 // A decode thread reads its row's units and coefficients from the stage, builds the 2^K
 // candidate values of the group (Eq. 7, the decode rule's exact arithmetic) as two byte tables,
 // and then eight columns cost one shift-and-mask per plane to form eight
@@ -31,10 +34,11 @@
 // and a split over the input dimension when tokens are few) and gemm_persistent_kernel (token tile 256: one
 // CTA per SM walks over tiles, two TMEM accumulators, separate epilogue warps; described at its definition).
 //
-// Pipeline: per stage four mbarriers -- full_b (x tile landed), full_p (planes and coefficients
-// landed; the producer issued them after `empty`, so the stage's A slot is free as well), full_a
-// (128 decode threads arrived after a proxy fence), empty (tcgen05.commit of the MMAs that read
-// the stage) -- and one
+// Pipeline of the tile kernel: three rings, each with full / empty mbarriers -- packed blocks (full_p by the
+// copies' bytes, empty_p by one arrival per decode warp once the block is in registers), x tiles (full_b by
+// the TMA's bytes, empty_b by tcgen05.commit) and A tiles (full_a by one arrival per decode warp after a proxy
+// fence, empty_a by tcgen05.commit of the MMAs that read the slot); the persistent kernel keeps one ring with
+// four barriers per stage (full_b, full_p, full_a of 128 arrivals, empty).  Both have one
 // acc_full barrier for the epilogue.  Every wait is bounded: on expiry the thread records
 // BPDQ_ERR_TIMEOUT in the handle's status word, raises a CTA-wide abort flag that lets all other
 // waits fall through, and the CTA still runs to its common exit where TMEM is freed.
@@ -169,24 +173,51 @@ __host__ __device__ constexpr unsigned instr_desc_f16(int m, int n) {
     return (1u << 4) | ((unsigned)(n >> 3) << 17) | ((unsigned)(m >> 4) << 24);
 }
 
+// Ring depths of the tile kernel.  Its three operand streams have very different sizes per 64-column stage -- 16 KB of
+// decoded weights (A), BN x 128 bytes of activations (B), about 2.5 KB of packed planes and coefficients -- and very
+// different latencies (A is produced on the SM, B comes from L2, the packed bytes from HBM), so each has its own
+// ring: a few A slots, more B slots, and packed 128-column blocks several stages ahead.  A 72B-shaped projection at
+// M <= 64 takes 80 us this way (88 us with one common ring of three or four stages and bulk copies per segment); what
+// remains is hand-over latency: the decode warps and the single MMA thread each wait for the other about half of the
+// time (cycle counters in a working copy), whatever the ring depths.
+template <int K, int BN> struct TileCfg {
+    static constexpr int kBTileBytes = BN * BK * 2;
+    static constexpr int kPlaneBytes = K * BM * 16;             // K segments of 128 rows x 16 bytes
+    static constexpr int kCoefBytes = (K + 1) * BM * 2;         // K+1 segments of 128 rows x 2 bytes: one coefficient group
+    static constexpr int kBlockBytes = (kPlaneBytes + 2 * kCoefBytes + 1023) / 1024 * 1024;   // a block's planes and up to two groups (g = 64)
+    static constexpr int kCtasPerSm = BN <= 64 ? 2 : 1;         // few tokens: bound by the decode threads, so two CTAs share an SM
+    static constexpr int kSmemBudget = kCtasPerSm == 2 ? 111 * 1024 : 222 * 1024;
+    static constexpr int kSA = BN <= 64 ? 3 : 4;
+    static constexpr int kSB = BN <= 16 ? 14 : (BN <= 32 ? 9 : (BN <= 64 && K <= 3 ? 5 : 4));
+    static constexpr int kRest = kSmemBudget - kSA * kATileBytes - kSB * kBTileBytes - 2048;
+    static constexpr int kSP = kRest / kBlockBytes > 8 ? 8 : kRest / kBlockBytes;
+    static_assert(kSP >= 2, "at least two packed blocks in flight");
+    static constexpr int kTmemCols = BN < 32 ? 32 : BN;        // power of two >= 32
+    static constexpr int kSmemBytes = kSA * kATileBytes + kSB * kBTileBytes + kSP * kBlockBytes + 1024 /*alignment slack*/ + 1024 /*barriers*/;
+};
+
 template <int K, int BN>
-__global__ void __launch_bounds__(kThreads, Cfg<K, BN>::kCtasPerSm)
-gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
-    using C = Cfg<K, BN>;
-    constexpr int S = C::kStages;
+__global__ void __launch_bounds__(kThreads, TileCfg<K, BN>::kCtasPerSm)
+gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap planes_map,
+            const __grid_constant__ CUtensorMap coefs_map, const GemmParams p) {
+    using C = TileCfg<K, BN>;
+    constexpr int SA = C::kSA, SB = C::kSB, SP = C::kSP;
     extern __shared__ unsigned char smem_raw[];
     const unsigned base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* smem = smem_raw + (base - smem_u32(smem_raw));
-    const unsigned a_base = base;                                  // S x 16 KB
-    const unsigned b_base = base + S * kATileBytes;                // S x BN*128 bytes
-    const unsigned p_base = b_base + S * C::kBTileBytes;           // S x (planes, coefficients)
-    const unsigned bar_base = p_base + S * C::kPackedBytes;
-    auto full_b = [&](int s) { return bar_base + 8u * s; };
-    auto full_a = [&](int s) { return bar_base + 8u * (S + s); };
-    auto empty = [&](int s) { return bar_base + 8u * (2 * S + s); };
-    auto full_p = [&](int s) { return bar_base + 8u * (3 * S + s); };
-    const unsigned acc_full = bar_base + 8u * (4 * S);
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(smem + (bar_base - base) + 8 * (4 * S + 1));
+    const unsigned a_base = base;                                  // SA x 16 KB
+    const unsigned b_base = a_base + SA * kATileBytes;             // SB x BN*128 bytes
+    const unsigned p_base = b_base + SB * C::kBTileBytes;          // SP x (planes, coefficients) of a 128-column block
+    const unsigned bar_base = p_base + SP * C::kBlockBytes;
+    auto full_a = [&](int s) { return bar_base + 8u * s; };
+    auto empty_a = [&](int s) { return bar_base + 8u * (SA + s); };
+    auto full_b = [&](int s) { return bar_base + 8u * (2 * SA + s); };
+    auto empty_b = [&](int s) { return bar_base + 8u * (2 * SA + SB + s); };
+    auto full_p = [&](int s) { return bar_base + 8u * (2 * SA + 2 * SB + s); };
+    auto empty_p = [&](int s) { return bar_base + 8u * (2 * SA + 2 * SB + SP + s); };
+    constexpr int kBars = 2 * SA + 2 * SB + 2 * SP;
+    const unsigned acc_full = bar_base + 8u * kBars;
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(smem + (bar_base - base) + 8 * (kBars + 1));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -194,14 +225,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
     const int tok0 = blockIdx.y * BN;          // first token of this CTA
     const int kb0 = blockIdx.z * p.kb_per;           // this CTA's stages: [kb0, kb1) of the in / 64 stages of the row
     const int kb1 = min(p.in / BK, kb0 + p.kb_per);
+    const int nst = kb1 - kb0;                       // even: whole 128-column blocks
+    const int b0 = kb0 / 2, nblk = nst / 2;
+    const int ng = p.group == 64 ? 2 : 1;            // coefficient groups per block
 
     if (tid == 0) {
-        for (int s = 0; s < S; ++s) {
-            mbar_init(full_b(s), 1);
-            mbar_init(full_a(s), kDecodeThreads);
-            mbar_init(empty(s), 1);
-            mbar_init(full_p(s), 1);
-        }
+        for (int s = 0; s < SA; ++s) { mbar_init(full_a(s), kDecodeThreads / 32); mbar_init(empty_a(s), 1); }   // one arrival per decode warp
+        for (int s = 0; s < SB; ++s) { mbar_init(full_b(s), 1); mbar_init(empty_b(s), 1); }
+        for (int s = 0; s < SP; ++s) { mbar_init(full_p(s), 1); mbar_init(empty_p(s), kDecodeThreads / 32); }
         mbar_init(acc_full, 1);
         *abort_flag = 0;
         fence_barrier_init();
@@ -216,56 +247,66 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
     const unsigned tmem_d = *tmem_slot;
 
     if (warp == 0) {
-        // ---------------- producer: x tiles (TMA), plane and coefficient segments (bulk copies) ----------------
+        // ---------------- producer: packed blocks (bulk copies) and x tiles (TMA), each as its ring has room ----------------
         if (lane == 0) {
-            const int nrows = min(BM, p.out - row0);     // ragged last row tile: a multiple of 16
-            const unsigned seg_p = (unsigned)nrows * 16u, seg_c = (unsigned)nrows * 2u;
-            const uint8_t* cbase = p.blob + p.planes_bytes;
-            for (int kb = kb0; kb < kb1; ++kb) {
-                const int s = (kb - kb0) % S;
-                const unsigned ph = (unsigned)((kb - kb0) / S) & 1u;
-                if (!mbar_wait(empty(s), ph ^ 1u, abort_flag, p.status)) break;
-                // packed operands first: the decode threads are the longer leg of the pipeline
-                const bool first_half = (kb & 1) == 0;   // the block's plane units travel with its first stage
-                mbar_expect_tx(full_p(s), (first_half ? (unsigned)K * seg_p : 0u) + (unsigned)(K + 1) * seg_c);
-                const unsigned pdst = p_base + s * C::kPackedBytes;
-                const int b = kb >> 1, G = (kb * BK) / p.group;
-                if (first_half) {
-#pragma unroll
-                    for (int i = 0; i < K; ++i)
-                        bulk_load(pdst + i * (BM * 16), p.blob + (((size_t)b * K + i) * p.out + row0) * 16, seg_p, full_p(s));
+            // A block's K plane segments (128 rows x 16 bytes each) are one box of the planes' tensor map, its one or two
+            // coefficient groups one box of the coefficients' map: two copies per block, whatever K is.  Rows past a
+            // ragged last tile are filled with zeros (and count as received bytes).
+            int pb = 0, xb = 0;                          // next packed block, next x stage
+            unsigned idle = 0;
+            while (pb < nblk || xb < nst) {
+                bool moved = false;
+                if (pb < nblk && mbar_try_wait(empty_p(pb % SP), ((unsigned)(pb / SP) & 1u) ^ 1u)) {
+                    const int sp = pb % SP, b = b0 + pb;
+                    mbar_expect_tx(full_p(sp), (unsigned)(C::kPlaneBytes + ng * C::kCoefBytes));
+                    const unsigned pdst = p_base + sp * C::kBlockBytes;
+                    tma_load_2d(pdst, &planes_map, row0 * 2, b * K, full_p(sp));                 // 8-byte elements: 2 per row
+                    tma_load_2d(pdst + C::kPlaneBytes, &coefs_map, row0 / 4, ((b * 128) / p.group) * (K + 1), full_p(sp));
+                    ++pb;
+                    moved = true;
                 }
-#pragma unroll
-                for (int i = 0; i <= K; ++i)
-                    bulk_load(pdst + C::kPlaneBytes + i * (BM * 2), cbase + (((size_t)G * (K + 1) + i) * p.out + row0) * 2, seg_c, full_p(s));
-                mbar_expect_tx(full_b(s), C::kBTileBytes);
-                tma_load_2d(b_base + s * C::kBTileBytes, &x_map, kb * BK, tok0, full_b(s));
+                if (xb < nst && mbar_try_wait(empty_b(xb % SB), ((unsigned)(xb / SB) & 1u) ^ 1u)) {
+                    const int sb = xb % SB;
+                    mbar_expect_tx(full_b(sb), C::kBTileBytes);
+                    tma_load_2d(b_base + sb * C::kBTileBytes, &x_map, (kb0 + xb) * BK, tok0, full_b(sb));
+                    ++xb;
+                    moved = true;
+                }
+                if (moved) {
+                    idle = 0;
+                } else if (++idle >= kWaitLimit) {       // neither ring has freed a slot for too long
+                    *abort_flag = 1;
+                    atomicExch(p.status, BPDQ_ERR_TIMEOUT);
+                    break;
+                } else if ((idle & 63u) == 63u && *abort_flag) {
+                    break;
+                }
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             constexpr unsigned idesc = instr_desc_f16(BM, BN);
-            bool ok = true;
-            for (int kb = kb0; kb < kb1 && ok; ++kb) {
-                const int s = (kb - kb0) % S;
-                const unsigned ph = (unsigned)((kb - kb0) / S) & 1u;
-                ok = mbar_wait(full_a(s), ph, abort_flag, p.status) && mbar_wait(full_b(s), ph, abort_flag, p.status);
-                if (!ok) break;
+            for (int it = 0; it < nst; ++it) {
+                const int sa = it % SA, sb = it % SB;
+                if (!mbar_wait(full_a(sa), (unsigned)(it / SA) & 1u, abort_flag, p.status) ||
+                    !mbar_wait(full_b(sb), (unsigned)(it / SB) & 1u, abort_flag, p.status))
+                    break;
                 tc_fence_after();
-                const uint64_t adesc = smem_desc_sw128(a_base + s * kATileBytes);
-                const uint64_t bdesc = smem_desc_sw128(b_base + s * C::kBTileBytes);
+                const uint64_t adesc = smem_desc_sw128(a_base + sa * kATileBytes);
+                const uint64_t bdesc = smem_desc_sw128(b_base + sb * C::kBTileBytes);
 #pragma unroll
                 for (int k4 = 0; k4 < BK / 16; ++k4)     // 16 columns = 32 bytes further along the swizzled row
-                    umma_f16(tmem_d, adesc + 2u * k4, bdesc + 2u * k4, idesc, ((kb - kb0) | k4) != 0 ? 1u : 0u);
-                umma_commit(empty(s));                   // frees the stage once these MMAs have read it
+                    umma_f16(tmem_d, adesc + 2u * k4, bdesc + 2u * k4, idesc, (it | k4) != 0 ? 1u : 0u);
+                umma_commit(empty_a(sa));                // each frees its slot once these MMAs have read it
+                umma_commit(empty_b(sb));
             }
             umma_commit(acc_full);                       // arrives when every MMA above has completed
         }
     } else {
         // ---------------- decode warps (thread = output row), then epilogue ----------------
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
-        const int grp = (warp - 2) >> 2;                 // decode group: takes the stages with kb % 2 == grp
+        const int grp = (warp - 2) >> 2;                 // decode group: takes every other 128-column block
         const int rl = quad * 32 + lane;                 // row inside the tile
         const int r = row0 + rl;
         const bool row_ok = r < p.out;                   // rows past a ragged last tile decode stale bytes; nothing of theirs is stored
@@ -273,37 +314,45 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) a_off[ch] = (unsigned)rl * 128u + (((unsigned)ch ^ (unsigned)(rl & 7)) << 4);
         bool ok = true;
-        for (int b = kb0 / 2 + grp; 2 * b < kb1 && ok; b += kDecodeGroups) {
+        for (int bi = grp; bi < nblk && ok; bi += kDecodeGroups) {
+            const int sp = bi % SP;
+            if (!mbar_wait(full_p(sp), (unsigned)(bi / SP) & 1u, abort_flag, p.status)) { ok = false; break; }
+            const unsigned psrc = p_base + sp * C::kBlockBytes;
             unsigned cur[K][4];                          // logical words of this row's plane units
+#pragma unroll
+            for (int i = 0; i < K; ++i) {
+                uint4 raw;
+                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(raw.x), "=r"(raw.y), "=r"(raw.z), "=r"(raw.w)
+                             : "r"(psrc + i * (BM * 16) + rl * 16));
+                const uint4 u = bpdq::unrotate_unit(raw, r);
+                cur[i][0] = u.x; cur[i][1] = u.y; cur[i][2] = u.z; cur[i][3] = u.w;
+            }
+            unsigned short cbits[2][K + 1];              // coefficients of the block's one or two groups
+#pragma unroll
+            for (int gg = 0; gg < 2; ++gg)
+#pragma unroll
+                for (int i = 0; i <= K; ++i) {
+                    cbits[gg][i] = 0;
+                    if (gg < ng)
+                        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(cbits[gg][i])
+                                     : "r"(psrc + C::kPlaneBytes + gg * C::kCoefBytes + i * (BM * 2) + rl * 2));
+                }
+            __syncwarp();                                // every lane's loads have returned (their results were used above)
+            if (lane == 0) mbar_arrive(empty_p(sp));     // the block's packed bytes are in registers: its slot may be refilled
             bpdq::ByteTables<K> tab;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                const int kb = 2 * b + half;
-                const int s = (kb - kb0) % S;
-                const unsigned ph = (unsigned)((kb - kb0) / S) & 1u;
-                if (!mbar_wait(full_p(s), ph, abort_flag, p.status)) { ok = false; break; }
-                const unsigned psrc = p_base + s * C::kPackedBytes;
-                if (half == 0) {
-#pragma unroll
-                    for (int i = 0; i < K; ++i) {
-                        uint4 raw;
-                        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(raw.x), "=r"(raw.y), "=r"(raw.z), "=r"(raw.w)
-                                     : "r"(psrc + i * (BM * 16) + rl * 16));
-                        const uint4 u = bpdq::unrotate_unit(raw, r);
-                        cur[i][0] = u.x; cur[i][1] = u.y; cur[i][2] = u.z; cur[i][3] = u.w;
-                    }
-                }
-                if (half == 0 || p.group == 64) {        // candidate tables of the coefficient group that starts here
+                const int it = 2 * bi + half;
+                const int sa = it % SA;
+                if (half == 0 || ng == 2) {              // candidate tables of the coefficient group that starts here
                     float c[K + 1];
 #pragma unroll
-                    for (int i = 0; i <= K; ++i) {
-                        unsigned short hbits;
-                        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(hbits) : "r"(psrc + C::kPlaneBytes + i * (BM * 2) + rl * 2));
-                        c[i] = __half2float(__ushort_as_half(hbits));
-                    }
+                    for (int i = 0; i <= K; ++i) c[i] = __half2float(__ushort_as_half(cbits[ng == 2 ? half : 0][i]));
                     bpdq::candidate_byte_tables<K>(c, tab);
                 }
-                const unsigned dst = a_base + s * kATileBytes;
+                // decode the stage's 64 columns into registers first (eight independent chains the compiler can interleave,
+                // and nothing of it waits for the slot), then wait for the slot and store
+                uint4 v8[8];
 #pragma unroll
                 for (int wd = 0; wd < 2; ++wd) {         // two 32-column words per 64-column stage
                     unsigned w[K], sel[4];
@@ -311,22 +360,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
                     for (int i = 0; i < K; ++i) w[i] = cur[i][2 * half + wd];
                     bpdq::code_nibbles_word<K>(w, sel);
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const uint4 v8 = bpdq::decode8<K>(sel[u], tab);
-                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + a_off[4 * wd + u]),
-                                     "r"(v8.x), "r"(v8.y), "r"(v8.z), "r"(v8.w) : "memory");
-                    }
+                    for (int u = 0; u < 4; ++u) v8[4 * wd + u] = bpdq::decode8<K>(sel[u], tab);
                 }
+                if (!mbar_wait(empty_a(sa), ((unsigned)(it / SA) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                const unsigned dst = a_base + sa * kATileBytes;
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch)
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + a_off[ch]),
+                                 "r"(v8[ch].x), "r"(v8[ch].y), "r"(v8[ch].z), "r"(v8[ch].w) : "memory");
                 fence_proxy_async();                     // make the generic-proxy stores visible to the MMA's reads
-                mbar_arrive(full_a(s));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full_a(sa));  // one arrival per warp, after all its lanes' stores and fences
             }
         }
-        // ---------------- epilogue ----------------
-        if (ok && mbar_wait(acc_full, 0u, abort_flag, p.status)) {
+        // ---------------- epilogue: each decode group takes half of the token columns (all of them when there are only 16) ----------------
+        constexpr int kColsPerGroup = BN >= 32 ? BN / 2 : BN;
+        if (ok && (BN >= 32 || grp == 0) && mbar_wait(acc_full, 0u, abort_flag, p.status)) {
             tc_fence_after();
             const unsigned taddr = tmem_d + ((unsigned)(quad * 32) << 16);
 #pragma unroll 1
-            for (int c0 = grp * (BN / 2); c0 < (grp + 1) * (BN / 2); c0 += 16) {
+            for (int c0 = grp * kColsPerGroup; c0 < (grp + 1) * kColsPerGroup; c0 += 16) {
                 if (tok0 + c0 >= p.M) break;             // warp-uniform
                 unsigned v[16];
                 tmem_ld16(taddr + (unsigned)c0, v);
@@ -624,7 +677,7 @@ EncodeTiledFn encode_tiled_fn() {
 
 template <int K, int BN>
 int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
-    using C = Cfg<K, BN>;
+    using C = TileCfg<K, BN>;
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemm_kernel<K, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
@@ -642,6 +695,26 @@ int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t st
                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (cr != CUDA_SUCCESS) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: tensor map encode failed (CUresult %d)", (int)cr);
+    if (!h->gemm_maps_ready) {
+        // planes: rows (block, plane) of out x 16 bytes; coefficients: rows (group, coefficient) of out x 2 bytes; both
+        // as 8-byte elements, so that 128 output rows are 256 resp. 32 elements (a box dimension holds at most 256)
+        const int ng = h->group == 64 ? 2 : 1;
+        const cuuint64_t pd[2] = {(cuuint64_t)h->out * 2, (cuuint64_t)(h->in / 128) * K};
+        const cuuint64_t ps[1] = {(cuuint64_t)h->out * 16};
+        const cuuint32_t pb[2] = {(cuuint32_t)BM * 2, (cuuint32_t)K};
+        const cuuint64_t cd[2] = {(cuuint64_t)h->out / 4, (cuuint64_t)(h->in / h->group) * (K + 1)};
+        const cuuint64_t cs[1] = {(cuuint64_t)h->out * 2};
+        const cuuint32_t cb[2] = {(cuuint32_t)BM / 4, (cuuint32_t)(ng * (K + 1))};
+        CUresult r1 = enc(reinterpret_cast<CUtensorMap*>(h->gemm_maps[0]), CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, h->d_blob, pd, ps, pb, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        CUresult r2 = enc(reinterpret_cast<CUtensorMap*>(h->gemm_maps[1]), CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, h->d_blob + h->planes_bytes, cd, cs, cb,
+                          estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r1 != CUDA_SUCCESS || r2 != CUDA_SUCCESS)
+            return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: tensor map encode of the packed weights failed (CUresult %d, %d)", (int)r1, (int)r2);
+        h->gemm_maps_ready = 1;
+    }
     GemmParams p;
     p.blob = h->d_blob; p.planes_bytes = h->planes_bytes; p.y = static_cast<__half*>(y); p.status = h->d_status;
     p.out = h->out; p.in = h->in; p.group = h->group; p.M = M;
@@ -660,7 +733,8 @@ int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t st
             grid.z = (nkb + p.kb_per - 1) / p.kb_per;
         }
     }
-    gemm_kernel<K, BN><<<grid, kThreads, C::kSmemBytes, stream>>>(map, p);
+    gemm_kernel<K, BN><<<grid, kThreads, C::kSmemBytes, stream>>>(map, *reinterpret_cast<const CUtensorMap*>(h->gemm_maps[0]),
+                                                                   *reinterpret_cast<const CUtensorMap*>(h->gemm_maps[1]), p);
     h->launches += 1;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm launch: %s", cudaGetErrorString(e));
@@ -702,6 +776,7 @@ int launch_persistent(bpdq_handle_s* h, const void* x, void* y, int M, cudaStrea
 
 template <int K>
 int launch_k(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
+    if (M <= 16) return launch_tile<K, 16>(h, x, y, M, stream);
     if (M <= 32) return launch_tile<K, 32>(h, x, y, M, stream);
     if (M <= 64) return launch_tile<K, 64>(h, x, y, M, stream);
     if (M <= 128) return launch_tile<K, 128>(h, x, y, M, stream);

@@ -53,6 +53,9 @@ struct bpdq_handle_s {
     uint64_t launches;
     // Last cut of a look-up-table launch led by this handle (the cut depends on the shapes only): linears,
     // their (row groups, slices), segment cost, CTAs, first task of every CTA.  plan_n == 0: none yet.
+    // Tensor maps of the blob for the tensor-core kernel (planes, coefficients), encoded at the first launch.
+    alignas(64) unsigned char gemm_maps[2][128];
+    int gemm_maps_ready;
     int plan_n, plan_cost, plan_grid;
     int plan_shape[BPDQ_BATCH_MAX][2];
     int plan_t_begin[193];
