@@ -27,6 +27,9 @@ pytestmark = pytest.mark.gpu
     (4, 128, 384, 2048, 7),      # two-way split, ragged token tile
     (2, 128, 256, 384, 20500),   # 162 output tiles for 148 persistent CTAs: a second tile per CTA, odd number of blocks per tile
     (4, 128, 128, 640, 38000),   # 149 tiles, three-stage ring (K = 4), odd number of blocks per tile
+    (3, 64, 160, 640, 24),       # tile kernel, ragged last row tile (the tensor maps fill the missing rows), two groups per block
+    (1, 256, 144, 1024, 100),    # tile kernel with the 128-token tile, ragged row tile, a group every two blocks
+    (2, 128, 400, 1152, 9),      # 16-token tile, odd number of blocks, rings wrap at different stages
 ])
 def test_gemm_kernel(K, g, out, in_, M):
     h, bits, coef = G.make_layer(60 + K, out, in_, K, g, max_M=M)
