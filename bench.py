@@ -303,7 +303,9 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
                        "l2": f"inputs larger than L2: {copies} distinct layer copies of {bytes_step / 1e6:.1f} MB rotated between steps",
                        "useful_bytes_per_step": bytes_step, "parallelism": "replicas only" if world > 1 else "single GPU"},
             "e2e": {"value": e2e_value, "unit": UNIT,
-                    "h2d_bytes_per_step": sum(2 * M * i for _, _, i in shapes), "d2h_bytes_per_step": sum(2 * M * o for _, o, _ in shapes)},
+                    "h2d_bytes_per_step": sum(2 * M * i for _, _, i in shapes), "d2h_bytes_per_step": sum(2 * M * o for _, o, _ in shapes),
+                    "path": "bpdq_linear_batch_host, every step: one gather launch reads the seven x from pinned host memory, the kernel "
+                            "stores the seven y into pinned host memory, one stream wait"},
             "gpu_launches": n_launch, "clocks": clocks,
             "roofline": {"bound": "hbm", "kernel": "gemv_lut_kernel", "achieved": per_gpu, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": per_gpu / peaks["hbm_gbs"], "peak_source": peaks["source"],

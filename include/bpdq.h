@@ -144,16 +144,19 @@ BPDQ_API int bpdq_linear_ex(bpdq_handle_t h, const void* x_fp16_dev, void* y_fp1
 BPDQ_API int bpdq_linear_batch(const bpdq_handle_t* hs, const void* const* xs_fp16_dev, void* const* ys_fp16_dev, int n,
                       int M, void* stream);
 
-/* bpdq_linear_batch for callers whose activations live in HOST memory: copies every x[k] (host, [M][in_k]) to
- * its handle's staging buffer, runs bpdq_linear_batch, copies every y[k] back to host memory and waits for
- * the stream once.  Same argument rules as bpdq_linear_batch; pinned host memory keeps the copies
- * asynchronous up to the final wait. */
+/* bpdq_linear_batch for callers whose activations live in HOST memory: brings every x[k] (host, [M][in_k])
+ * into its handle's staging buffer, runs bpdq_linear_batch, returns every y[k] to host memory and waits for
+ * the stream once.  Same argument rules as bpdq_linear_batch.  When every buffer is pinned (page-locked)
+ * and 16-byte aligned, one gather kernel reads all x through their device-visible addresses and the
+ * look-up-table kernel stores y straight into host memory: two launches and one wait per call.  Pageable
+ * or unaligned buffers take one copy per buffer and direction instead. */
 BPDQ_API int bpdq_linear_batch_host(const bpdq_handle_t* hs, const void* const* xs_fp16_host, void* const* ys_fp16_host, int n,
                            int M, void* stream);
 
 /* Same map for callers whose activations live in HOST memory: copies x (host, [M][in]) to a
  * handle-owned staging buffer, runs bpdq_linear, copies y back to `y_fp16_host` and waits for
- * the stream.  Pinned host memory makes the copies asynchronous up to that wait. */
+ * the stream.  Pinned host memory makes the copies asynchronous up to that wait; token counts that
+ * go to the look-up-table kernel take bpdq_linear_batch_host's path with n = 1. */
 BPDQ_API int bpdq_linear_host(bpdq_handle_t h, const void* x_fp16_host, void* y_fp16_host, int M,
                      void* stream);
 

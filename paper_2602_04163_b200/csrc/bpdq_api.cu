@@ -27,6 +27,34 @@ void free_handle(bpdq_handle_s* h) {
     delete h;
 }
 
+// Activations of up to BPDQ_BATCH_MAX linears from pinned host memory into the handles' staging buffers, one launch:
+// the kernel reads the host buffers through their device-visible addresses, sixteen bytes per thread and access.
+struct GatherParams {
+    const uint4* src[BPDQ_BATCH_MAX];
+    uint4* dst[BPDQ_BATCH_MAX];
+    unsigned end16[BPDQ_BATCH_MAX];     // running end of every buffer, in 16-byte units
+    int n;
+};
+__global__ void gather_kernel(const __grid_constant__ GatherParams p) {
+    const unsigned total = p.end16[p.n - 1];
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        int k = 0;
+        while (i >= p.end16[k]) ++k;
+        const unsigned j = i - (k ? p.end16[k - 1] : 0u);
+        p.dst[k][j] = p.src[k][j];
+    }
+}
+
+// Device-visible address of a pinned (page-locked) host buffer; null for pageable or foreign memory.
+void* mapped_address(const void* host) {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, host) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
+}
+
 int check_linear_args(bpdq_handle_s* h, const void* x, void* y, int M, const char* who) {
     if (!h) return set_error(BPDQ_ERR_INVALID, "%s: null handle", who);
     if (M < 0 || M > h->max_M) return set_error(BPDQ_ERR_INVALID, "%s: M=%d outside [0, max_M=%d]", who, M, h->max_M);
@@ -173,6 +201,8 @@ extern "C" int bpdq_linear(bpdq_handle_t h, const void* x, void* y, int M, void*
 extern "C" int bpdq_linear_host(bpdq_handle_t h, const void* x_host, void* y_host, int M, void* stream) {
     int rc = check_linear_args(h, x_host, y_host, M, "bpdq_linear_host");
     if (rc != BPDQ_OK || M == 0) return rc;
+    if (M <= h->gemv_max_m && M <= BPDQ_GEMV_MAX_M && gemv_supported(h->out, h->in, h->K, h->group))
+        return bpdq_linear_batch_host(&h, &x_host, &y_host, 1, M, stream);      // the look-up-table kernel: same path as a batch of one
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(h->d_xstage, x_host, (size_t)M * h->in * 2, cudaMemcpyHostToDevice, s);
     if (e != cudaSuccess) return cuda_fail("bpdq_linear_host: copy in", e);
@@ -198,6 +228,39 @@ extern "C" int bpdq_linear_batch_host(const bpdq_handle_t* hs, const void* const
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const void* xd[BPDQ_BATCH_MAX];
     void* yd[BPDQ_BATCH_MAX];
+    // Pinned, 16-byte aligned host buffers: one gather launch brings every x into its staging buffer, and the kernel
+    // writes every y straight into host memory (its stores are posted, nobody waits for them), so a step is two
+    // launches and one wait instead of 2n copies.  Anything else takes the copy path below.
+    {
+        GatherParams g;
+        g.n = n;
+        bool direct = true;
+        unsigned end16 = 0;
+        for (int k = 0; k < n && direct; ++k) {
+            void* xm = mapped_address(xs_host[k]);
+            void* ym = mapped_address(ys_host[k]);
+            direct = xm && ym && aligned16(xm) && aligned16(ym);
+            g.src[k] = static_cast<const uint4*>(xm);
+            g.dst[k] = static_cast<uint4*>(hs[k]->d_xstage);
+            end16 += (unsigned)((size_t)M * hs[k]->in * 2 / 16);        // in is a multiple of 128: whole 16-byte units
+            g.end16[k] = end16;
+            xd[k] = hs[k]->d_xstage;
+            yd[k] = ym;
+        }
+        if (direct) {
+            unsigned blocks = (end16 + 255u) / 256u;
+            if (blocks > 148u) blocks = 148u;
+            gather_kernel<<<blocks, 256, 0, s>>>(g);
+            hs[0]->launches += 1;
+            cudaError_t e = cudaGetLastError();
+            if (e != cudaSuccess) return cuda_fail("bpdq_linear_batch_host: gather launch", e);
+            const int rc = bpdq_linear_batch(hs, xd, yd, n, M, stream);
+            if (rc != BPDQ_OK) return rc;
+            e = cudaStreamSynchronize(s);
+            if (e != cudaSuccess) return cuda_fail("bpdq_linear_batch_host: synchronize", e);
+            return BPDQ_OK;
+        }
+    }
     for (int k = 0; k < n; ++k) {
         cudaError_t e = cudaMemcpyAsync(hs[k]->d_xstage, xs_host[k], (size_t)M * hs[k]->in * 2, cudaMemcpyHostToDevice, s);
         if (e != cudaSuccess) return cuda_fail("bpdq_linear_batch_host: copy in", e);

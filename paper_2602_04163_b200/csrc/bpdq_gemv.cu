@@ -57,7 +57,7 @@ struct GemvLinear {
 constexpr int kMaxBatch = BPDQ_BATCH_MAX;
 constexpr int kMaxGrid = 192;                        // CTAs of a launch (one per SM)
 // set-up and hand-over of one (slice, row range) segment, in tasks; measured optima for one / several linears per launch
-constexpr int kSegmentCostSingle = 32, kSegmentCostBatch = 48;
+constexpr int kSegmentCostSingle = 64, kSegmentCostBatch = 48;
 
 struct GemvParams {
     GemvLinear lin[kMaxBatch];

@@ -100,3 +100,37 @@ def test_batch_host_buffers_match_device_call():
     binding.bpdq_linear_batch_host(handles, [x.data_ptr() for x in xh], [y.data_ptr() for y in yh], M, G.stream_ptr())
     for y, w in zip(yh, want):
         assert np.allclose(y.numpy().astype(np.float64), w, rtol=2.0 ** -9, atol=1e-5)
+
+
+@pytest.mark.parametrize("pinned,M", [(True, 1), (True, 3), (False, 2)])
+def test_batch_host_buffers_pinned_and_pageable(pinned, M):
+    """Pinned buffers go through the gather launch with y stored straight into host memory (M = 3: two passes of the
+    kernel); pageable ones through one copy per buffer.  Both must give what the device call gives."""
+    K, g = 3, 128
+    shapes = [(160, 640), (400, 1152)]
+    layers = [G.make_layer(290 + k, o, i, K, g, max_M=M) for k, (o, i) in enumerate(shapes)]
+    handles = [L[0] for L in layers]
+    xs = [synth.activations(291 + k, M, i) for k, (_, i) in enumerate(shapes)]
+    want = _run_batch(handles, xs, M)
+    xh = [torch.from_numpy(x.view(np.int16).copy()).view(torch.float16) for x in xs]
+    yh = [torch.full((M, o), float("nan"), dtype=torch.float16) for o, _ in shapes]
+    if pinned:
+        xh, yh = [x.pin_memory() for x in xh], [y.pin_memory() for y in yh]
+    for _ in range(2):                                   # the second call finds the workspace as the first left it
+        binding.bpdq_linear_batch_host(handles, [x.data_ptr() for x in xh], [y.data_ptr() for y in yh], M, G.stream_ptr())
+        for y, w in zip(yh, want):
+            assert np.allclose(y.numpy().astype(np.float64), w, rtol=2.0 ** -9, atol=1e-5)
+            y.fill_(float("nan"))
+
+
+@pytest.mark.parametrize("M", [1, 40])
+def test_single_host_call(M):
+    """bpdq_linear_host: one token takes the look-up-table kernel's host path, forty tokens the copies around the tensor-core kernel."""
+    K, g, out, in_ = 2, 128, 272, 896
+    h, bits, coef = G.make_layer(310, out, in_, K, g, max_M=M)
+    x = synth.activations(311, M, in_)
+    want = G.run_linear(h, x, binding.KERNEL_AUTO)
+    xh = torch.from_numpy(x.view(np.int16).copy()).view(torch.float16).pin_memory()
+    yh = torch.full((M, out), float("nan"), dtype=torch.float16).pin_memory()
+    h.bpdq_linear_host(xh.data_ptr(), yh.data_ptr(), M, G.stream_ptr())
+    assert np.allclose(yh.numpy().astype(np.float64), want.astype(np.float64), rtol=2.0 ** -9, atol=1e-5)
