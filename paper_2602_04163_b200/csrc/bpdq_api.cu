@@ -36,6 +36,9 @@ struct GatherParams {
     int n;
 };
 __global__ void gather_kernel(const __grid_constant__ GatherParams p) {
+    // the look-up-table kernel behind it may take the free SMs and request its first weights at once; it reads x only
+    // after its own griddepcontrol.wait, i.e. after this kernel has finished
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const unsigned total = p.end16[p.n - 1];
     for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
         int k = 0;
@@ -248,9 +251,10 @@ extern "C" int bpdq_linear_batch_host(const bpdq_handle_t* hs, const void* const
             yd[k] = ym;
         }
         if (direct) {
-            unsigned blocks = (end16 + 255u) / 256u;
-            if (blocks > 148u) blocks = 148u;
-            gather_kernel<<<blocks, 256, 0, s>>>(g);
+            // few, full CTAs: every thread has about one access in flight, and most SMs stay free for the kernel behind
+            unsigned blocks = (end16 + 1023u) / 1024u;
+            if (blocks > 64u) blocks = 64u;
+            gather_kernel<<<blocks, 1024, 0, s>>>(g);
             hs[0]->launches += 1;
             cudaError_t e = cudaGetLastError();
             if (e != cudaSuccess) return cuda_fail("bpdq_linear_batch_host: gather launch", e);
