@@ -12,8 +12,8 @@
 // 16-byte chunk c of row r is stored at chunk position c ^ (r mod 8).  TMA writes that layout by
 // itself; the decode threads reproduce it by hand.
 //
-// Roles (320 threads): warp 0 is the producer (one lane: TMA loads of x and of the packed weights);
-// warp 1 allocates TMEM and issues the MMAs (one lane); warps 2..9 decode in two groups of four
+// Roles (320 threads; the tile kernel has a second MMA-issuing warp, 352): warp 0 is the producer (one lane: TMA
+// loads of x and of the packed weights); warp 1 allocates TMEM and issues the MMAs (one lane); eight warps decode in two groups of four
 // warps, thread = output row, group 0 taking the even 128-column blocks (two stages each) and
 // group 1 the odd ones (one warp per scheduler could not hide its own instruction latencies).
 // The packed planes and coefficients come through the pipeline as well, so that no decode thread
@@ -55,6 +55,7 @@ constexpr int BK = 64;                  // columns per stage: one 128-byte swizz
 constexpr int kDecodeGroups = 2;
 constexpr int kDecodeThreads = 128;               // per group: one thread per output row
 constexpr int kThreads = 64 + kDecodeGroups * kDecodeThreads;
+constexpr int kTileThreads = 96 + kDecodeGroups * kDecodeThreads;   // tile kernel: producer warp, two MMA-issuing warps, eight decode warps
 constexpr int kATileBytes = BM * BK * 2;                       // 16 KB
 constexpr unsigned kWaitLimit = 1u << 24;                      // polls of try_wait before a wait gives up
 
@@ -187,21 +188,29 @@ template <int K, int BN> struct TileCfg {
     static constexpr int kBlockBytes = (kPlaneBytes + 2 * kCoefBytes + 1023) / 1024 * 1024;   // a block's planes and up to two groups (g = 64)
     static constexpr int kCtasPerSm = BN <= 64 ? 2 : 1;         // few tokens: bound by the decode threads, so two CTAs share an SM
     static constexpr int kSmemBudget = kCtasPerSm == 2 ? 111 * 1024 : 222 * 1024;
-    static constexpr int kSA = BN <= 64 ? 3 : 4;
-    static constexpr int kSB = BN <= 16 ? 14 : (BN <= 32 ? 9 : (BN <= 64 && K <= 3 ? 5 : 4));
+    // One thread issues a tcgen05.mma every 160 clocks or so whatever its shape, while the pipe could take one of these
+    // few-column MMAs every 40 to 50 clocks: up to 32 tokens two warps issue, stage `it` going to issuer it % 2, each into
+    // an accumulator of its own (added up in the epilogue).  A parity wait is only safe on consecutive phases, so every
+    // barrier must always be waited on by the same thread or group: the ring lengths are multiples of the issuer count
+    // and of the number of decode groups (each group then owns two A slots and every other packed slot).
+    static constexpr int kIssuers = BN <= 32 ? 2 : 1;
+    static constexpr int kSA = kIssuers == 2 ? 4 : (BN <= 64 ? 3 : 4);
+    static constexpr int kSB = BN <= 16 ? 8 : (BN <= 32 ? (K <= 3 ? 6 : 4) : 4);
     static constexpr int kRest = kSmemBudget - kSA * kATileBytes - kSB * kBTileBytes - 2048;
-    static constexpr int kSP = kRest / kBlockBytes > 8 ? 8 : kRest / kBlockBytes;
+    static constexpr int kSP = (kRest / kBlockBytes > 8 ? 8 : kRest / kBlockBytes) / kDecodeGroups * kDecodeGroups;
     static_assert(kSP >= 2, "at least two packed blocks in flight");
-    static constexpr int kTmemCols = BN < 32 ? 32 : BN;        // power of two >= 32
+    static_assert(kSA % kIssuers == 0 && kSB % kIssuers == 0, "all uses of a slot go to one issuer");
+    static constexpr int kAccCols = kIssuers * BN;
+    static constexpr int kTmemCols = kAccCols <= 32 ? 32 : (kAccCols <= 64 ? 64 : (kAccCols <= 128 ? 128 : 256));   // power of two >= 32
     static constexpr int kSmemBytes = kSA * kATileBytes + kSB * kBTileBytes + kSP * kBlockBytes + 1024 /*alignment slack*/ + 1024 /*barriers*/;
 };
 
 template <int K, int BN>
-__global__ void __launch_bounds__(kThreads, TileCfg<K, BN>::kCtasPerSm)
+__global__ void __launch_bounds__(kTileThreads, TileCfg<K, BN>::kCtasPerSm)
 gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap planes_map,
             const __grid_constant__ CUtensorMap coefs_map, const GemmParams p) {
     using C = TileCfg<K, BN>;
-    constexpr int SA = C::kSA, SB = C::kSB, SP = C::kSP;
+    constexpr int SA = C::kSA, SB = C::kSB, SP = C::kSP, NI = C::kIssuers;
     extern __shared__ unsigned char smem_raw[];
     const unsigned base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* smem = smem_raw + (base - smem_u32(smem_raw));
@@ -233,7 +242,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
         for (int s = 0; s < SA; ++s) { mbar_init(full_a(s), kDecodeThreads / 32); mbar_init(empty_a(s), 1); }   // one arrival per decode warp
         for (int s = 0; s < SB; ++s) { mbar_init(full_b(s), 1); mbar_init(empty_b(s), 1); }
         for (int s = 0; s < SP; ++s) { mbar_init(full_p(s), 1); mbar_init(empty_p(s), kDecodeThreads / 32); }
-        mbar_init(acc_full, 1);
+        mbar_init(acc_full, NI);
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -283,11 +292,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
                 }
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+    } else if (warp <= 2) {
+        // ---------------- MMA issuers: warp 1 + j takes the stages it % NI == j, into accumulator j ----------------
+        if (lane == 0 && warp <= NI) {
             constexpr unsigned idesc = instr_desc_f16(BM, BN);
-            for (int it = 0; it < nst; ++it) {
+            const int j = warp - 1;
+            for (int it = j; it < nst; it += NI) {
                 const int sa = it % SA, sb = it % SB;
                 if (!mbar_wait(full_a(sa), (unsigned)(it / SA) & 1u, abort_flag, p.status) ||
                     !mbar_wait(full_b(sb), (unsigned)(it / SB) & 1u, abort_flag, p.status))
@@ -297,16 +307,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
                 const uint64_t bdesc = smem_desc_sw128(b_base + sb * C::kBTileBytes);
 #pragma unroll
                 for (int k4 = 0; k4 < BK / 16; ++k4)     // 16 columns = 32 bytes further along the swizzled row
-                    umma_f16(tmem_d, adesc + 2u * k4, bdesc + 2u * k4, idesc, (it | k4) != 0 ? 1u : 0u);
+                    umma_f16(tmem_d + (unsigned)(j * BN), adesc + 2u * k4, bdesc + 2u * k4, idesc, (it >= NI || k4 != 0) ? 1u : 0u);
                 umma_commit(empty_a(sa));                // each frees its slot once these MMAs have read it
                 umma_commit(empty_b(sb));
             }
-            umma_commit(acc_full);                       // arrives when every MMA above has completed
+            umma_commit(acc_full);                       // arrives when every MMA of this issuer has completed
         }
     } else {
         // ---------------- decode warps (thread = output row), then epilogue ----------------
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
-        const int grp = (warp - 2) >> 2;                 // decode group: takes every other 128-column block
+        const int grp = (warp - 3) >> 2;                 // decode group: takes every other 128-column block
         const int rl = quad * 32 + lane;                 // row inside the tile
         const int r = row0 + rl;
         const bool row_ok = r < p.out;                   // rows past a ragged last tile decode stale bytes; nothing of theirs is stored
@@ -381,16 +391,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
 #pragma unroll 1
             for (int c0 = grp * kColsPerGroup; c0 < (grp + 1) * kColsPerGroup; c0 += 16) {
                 if (tok0 + c0 >= p.M) break;             // warp-uniform
-                unsigned v[16];
-                tmem_ld16(taddr + (unsigned)c0, v);
-                tmem_ld_wait();
+                float acc[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+#pragma unroll
+                for (int a = 0; a < NI; ++a) {           // the issuers' accumulators, in a fixed order (every issuer has a stage: nst >= 2)
+                    unsigned v[16];
+                    tmem_ld16(taddr + (unsigned)(a * BN + c0), v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) acc[j] += __uint_as_float(v[j]);
+                }
                 if (row_ok) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const int t = tok0 + c0 + j;
                         if (t < p.M) {
-                            if (gridDim.z > 1) atomicAdd(p.ws + (size_t)t * p.out + r, __uint_as_float(v[j]));
-                            else p.y[(size_t)t * p.out + r] = __float2half_rn(__uint_as_float(v[j]));
+                            if (gridDim.z > 1) atomicAdd(p.ws + (size_t)t * p.out + r, acc[j]);
+                            else p.y[(size_t)t * p.out + r] = __float2half_rn(acc[j]);
                         }
                     }
                 }
@@ -416,7 +434,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
         if (*last) {
             __threadfence();
             const int ntok = min(BN, p.M - tok0);
-            for (int idx = tid; idx < ntok * BM; idx += kThreads) {
+            for (int idx = tid; idx < ntok * BM; idx += kTileThreads) {
                 const int t = tok0 + idx / BM, r = row0 + idx % BM;
                 if (r < p.out) {
                     float* src = p.ws + (size_t)t * p.out + r;
@@ -733,7 +751,7 @@ int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t st
             grid.z = (nkb + p.kb_per - 1) / p.kb_per;
         }
     }
-    gemm_kernel<K, BN><<<grid, kThreads, C::kSmemBytes, stream>>>(map, *reinterpret_cast<const CUtensorMap*>(h->gemm_maps[0]),
+    gemm_kernel<K, BN><<<grid, kTileThreads, C::kSmemBytes, stream>>>(map, *reinterpret_cast<const CUtensorMap*>(h->gemm_maps[0]),
                                                                    *reinterpret_cast<const CUtensorMap*>(h->gemm_maps[1]), p);
     h->launches += 1;
     cudaError_t e = cudaGetLastError();
