@@ -162,7 +162,7 @@ extern "C" int bpdq_linear_ex(bpdq_handle_t h, const void* x, void* y, int M, in
             if (M > BPDQ_GEMV_MAX_M)
                 return set_error(BPDQ_ERR_INVALID, "bpdq_linear: look-up-table kernel takes M <= %d, got %d", BPDQ_GEMV_MAX_M, M);
             if (!gemv_supported(h->out, h->in, h->K, h->group))
-                return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear: look-up-table kernel does not cover K=%d g=%d", h->K, h->group);
+                return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear: look-up-table kernel does not cover this linear (K=%d g=%d; packed weights must stay below 4 GB)", h->K, h->group);
             return launch_gemv(h, x, y, M, s);
         case BPDQ_KERNEL_GEMM:
             if (!gemm_supported(h->out, h->in, h->K, h->group))
@@ -187,7 +187,7 @@ extern "C" int bpdq_linear_batch(const bpdq_handle_t* hs, const void* const* xs,
         if ((hs[k]->group == 64) != (hs[0]->group == 64))
             return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: linear %d and linear 0 differ in having group 64", k);
         if (!gemv_supported(hs[k]->out, hs[k]->in, hs[k]->K, hs[k]->group))
-            return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear_batch: look-up-table kernel does not cover K=%d g=%d", hs[k]->K, hs[k]->group);
+            return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear_batch: look-up-table kernel does not cover linear %d (K=%d g=%d; packed weights must stay below 4 GB)", k, hs[k]->K, hs[k]->group);
         for (int j = 0; j < k; ++j)
             if (hs[j] == hs[k]) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: handle %d repeats handle %d", k, j);
         if (M > 0 && (!xs[k] || !ys[k] || !aligned16(xs[k]) || !aligned16(ys[k])))

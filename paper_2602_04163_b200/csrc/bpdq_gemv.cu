@@ -642,7 +642,11 @@ int launch_k(bpdq_handle_s* const* hs, GemvParams p, const void* const* xs, void
 
 namespace bpdq {
 
-bool gemv_supported(int, int, int K, int group) { return K >= 1 && K <= 4 && (group == 64 || group == 128 || group == 256); }
+// The kernel addresses the blob with 32-bit offsets: linears whose packed weights reach 4 GB go to the other kernels.
+bool gemv_supported(int out, int in, int K, int group) {
+    if (!(K >= 1 && K <= 4 && (group == 64 || group == 128 || group == 256))) return false;
+    return (unsigned long long)planes_bytes(out, in, K) + coefs_bytes(out, in, K, group) < (1ull << 32);
+}
 
 // binary32 row sums: kMaxMT tokens for the look-up-table kernel; up to 64 tokens for the tensor-core kernel's split
 // over the input dimension
