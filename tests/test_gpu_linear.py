@@ -1,6 +1,7 @@
 """bpdq_linear (all kernels) against the checker: |y - y_ref| <= 4e-3 * sum|x w| + 1e-3 per element."""
 import numpy as np
 import pytest
+import torch
 
 import oracle
 from paper_2602_04163_b200 import binding, synth
@@ -99,3 +100,30 @@ def test_lut_kernel_full_size_sampled(name, out, in_, K):
                                  synth.coefficients(900 + K, out, in_, K, g, rows), x, g)
     G.assert_linear_close(y[:, rows], y_ref, a_ref, name)
     assert np.all(np.isfinite(y))
+
+
+@pytest.mark.parametrize("M", [1, 2])
+def test_chain_of_dependent_launches(M):
+    """Three linears, each reading what the one before wrote, enqueued twice without a host wait in between.
+    The look-up-table kernel starts before the kernel in front of it has finished (it only requests weights that
+    early); every stage must still see the finished output of the stage before, and the second round must find
+    workspaces and counters as the first left them."""
+    K, g = 2, 128
+    dims = [(640, 384), (896, 640), (160, 896)]                     # (out, in): in of a stage is out of the one before
+    layers = [G.make_layer(400 + k, o, i, K, g, max_M=M) for k, (o, i) in enumerate(dims)]
+    x0 = G.x_tensor(synth.activations(410, M, dims[0][1]))
+    ys = [torch.full((M, o), float("nan"), dtype=torch.float16, device="cuda") for o, _ in dims]
+    sp = G.stream_ptr()
+    for _ in range(2):
+        src = x0
+        for (h, _, _), y in zip(layers, ys):
+            h.bpdq_linear_ex(src.data_ptr(), y.data_ptr(), M, binding.KERNEL_GEMV, sp)
+            src = y
+    torch.cuda.synchronize()
+    src = x0
+    for k, ((h, bits, coef), y) in enumerate(zip(layers, ys)):
+        h.bpdq_get_status(sp)
+        x_bits = src.cpu().view(torch.int16).numpy().view(np.uint16)
+        y_ref, a_ref = oracle.linear(bits, coef, x_bits, g)
+        G.assert_linear_close(y.cpu().numpy().astype(np.float64), y_ref, a_ref, f"stage {k}")
+        src = y
