@@ -28,6 +28,7 @@
 // last contribution to round those rows to binary16, write y and zero the workspace again.
 // Algorithmic HBM bytes per weight: K/8 + 2(K+1)/g.
 #include "bpdq_internal.h"
+#include "bpdq_partition.h"
 
 #include <cuda_fp16.h>
 
@@ -536,8 +537,7 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     // Cut the task space into one contiguous share per SM such that the most expensive share is as
     // cheap as possible, a segment (a CTA's visit to one slice of one linear: table set-up, drain,
     // hand-over) counting as kSegmentCost tasks.  Short slices (few output rows) would otherwise load
-    // the CTAs that get them with many set-ups.  The smallest feasible bound is found by bisection: for
-    // a given bound every CTA in turn takes as many tasks as fit under it.
+    // the CTAs that get them with many set-ups.  The cut itself is plain host code (bpdq_partition.h).
     int grid = h->sm_count < kMaxGrid ? h->sm_count : kMaxGrid;
     if ((long long)grid > total) grid = (int)total;
     const int kSegmentCost = p.n > 1 ? kSegmentCostBatch : kSegmentCostSingle;
@@ -547,39 +547,9 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     if (cached) {
         for (int c = 0; c <= grid; ++c) p.t_begin[c] = h->plan_t_begin[c];
     } else {
-        constexpr int kMinSegment = 8;                // a share is closed rather than opened into a slice for fewer tasks than this
-        // fills t_begin for the bound; true when `grid` shares cover the task space
-        auto sweep = [&](const double bound) {
-            long long t = 0;
-            int k = 0, b = 0;
-            p.t_begin[0] = 0;
-            while (t < total && b < grid) {
-                double budget = bound;
-                const long long start = t;
-                while (t < total) {
-                    while (k + 1 < p.n && t >= p.lin[k + 1].task_begin) ++k;
-                    const long long in_slice = p.lin[k].nrg - (t - p.lin[k].task_begin) % p.lin[k].nrg;   // tasks left in the current slice
-                    const double room = budget - kSegmentCost;
-                    if (t > start && room < (double)(in_slice < kMinSegment ? in_slice : kMinSegment)) break;
-                    long long take = room >= 1.0 ? (long long)room : 1;
-                    if (take > in_slice) take = in_slice;
-                    t += take;
-                    budget -= (double)(kSegmentCost + take);
-                    if (take < in_slice) break;
-                }
-                p.t_begin[++b] = (int)t;
-            }
-            const bool covered = t >= total;
-            for (int c = b + 1; c <= grid; ++c) p.t_begin[c] = (int)total;
-            return covered;
-        };
-        double lo = (double)total / grid, hi = 2.0 * (double)total / grid + 16.0 * kSegmentCost + 16.0;
-        while (!sweep(hi)) hi *= 2.0;                 // terminates: a bound above the whole cost covers everything
-        for (int it = 0; it < 24 && hi - lo > 0.5; ++it) {
-            const double mid = 0.5 * (lo + hi);
-            if (sweep(mid)) hi = mid; else lo = mid;
-        }
-        sweep(hi);
+        int nrg[kMaxBatch], nsl[kMaxBatch];
+        for (int k = 0; k < p.n; ++k) { nrg[k] = p.lin[k].nrg; nsl[k] = p.lin[k].nslices; }
+        bpdq::cut_task_space(nrg, nsl, p.n, grid, kSegmentCost, p.t_begin);
         h->plan_n = p.n; h->plan_cost = kSegmentCost; h->plan_grid = grid;
         for (int k = 0; k < p.n; ++k) { h->plan_shape[k][0] = p.lin[k].nrg; h->plan_shape[k][1] = p.lin[k].nslices; }
         for (int c = 0; c <= grid; ++c) h->plan_t_begin[c] = p.t_begin[c];
