@@ -541,6 +541,20 @@ def full_stack_section(torch, binding, peaks, sp, stream, n_layers=80):
     b = n_layers * layer_bytes(shapes, K, 1)
     res = {"layers": n_layers, "linears": len(hs), "packed_gb": sum(h.packed_bytes for h in hs) / 1e9, "ms_per_sweep": ms,
            "gbs": b / (ms * 1e-3) / 1e9, "frac_measured": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+    # the same sweep as one bpdq_linear_batch call per layer (every linear of a batch needs an output of its own)
+    n = len(shapes)
+    ys_each = [torch.empty((1, o), dtype=torch.float16, device="cuda") for _, o, _ in shapes]
+    x_ptrs = [xs[i].data_ptr() for _, _, i in shapes]
+    y_ptrs = [y.data_ptr() for y in ys_each]
+
+    def sweep_batched():
+        for layer in range(n_layers):
+            binding.bpdq_linear_batch(hs[layer * n:(layer + 1) * n], x_ptrs, y_ptrs, 1, sp)
+    sweep_batched()
+    ms_b = sorted(event_time_ms(torch, sweep_batched, stream) for _ in range(3))[1]
+    res["one_launch_per_layer"] = {"launches": n_layers, "ms_per_sweep": ms_b, "gbs": b / (ms_b * 1e-3) / 1e9,
+                                   "frac_measured": b / (ms_b * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     for h in hs:
         h.bpdq_destroy()
     return res
