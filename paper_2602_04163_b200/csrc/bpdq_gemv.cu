@@ -74,7 +74,12 @@ struct GemvParams {
 template <int K, int NG>
 struct Task {
     uint4 pl[2][K];
-    unsigned short cf[2][NG][K + 1];     // NG coefficient groups per 128-column block (two when g = 64)
+    unsigned short cf[2][K + 1];         // g >= 128: this row's coefficients of the block's group
+    // g = 64 (NG = 2): two groups per block would double the registers a task in flight holds, so a lane pair shares
+    // the loads: rows r (even lane) and r + 1 are adjacent in the blob, the even lane loads both rows' coefficients of
+    // the block's first group as 32-bit words, the odd lane those of the second group, and they swap halves by shuffle
+    // when the task is processed.
+    unsigned cfp[2][NG == 2 ? K + 1 : 1];
 };
 
 __device__ __forceinline__ uint4 ldg_stream16(const uint8_t* p) {
@@ -87,6 +92,11 @@ __device__ __forceinline__ uint4 ldg_stream16(const uint8_t* p) {
 __device__ __forceinline__ unsigned ldg_first4(const void* p) {
     unsigned v;
     asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ unsigned ldg_stream4(const uint8_t* p) {
+    unsigned v;
+    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
     return v;
 }
 __device__ __forceinline__ unsigned short ldg_stream2(const uint8_t* p) {
@@ -292,17 +302,21 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
 #pragma unroll
                     for (int i = 0; i < K; ++i) tk.pl[q][i] = ldg_stream16(L.blob + (size_t)(ps + i * plane_pitch));
                     const unsigned cs = csrc[q] + (unsigned)n * (W * 32);
+                    if constexpr (NG == 2) {          // the pair's even row, group a & 1 (rows are even-aligned: out is a multiple of 16)
+                        const unsigned cp = cs - 2u * (a & 1) + (unsigned)(a & 1) * (K + 1) * coef_pitch;
 #pragma unroll
-                    for (int gg = 0; gg < NG; ++gg)
+                        for (int i = 0; i <= K; ++i) tk.cfp[q][i] = ldg_stream4(L.blob + (size_t)(cp + i * coef_pitch));
+                    } else {
 #pragma unroll
-                        for (int i = 0; i <= K; ++i) tk.cf[q][gg][i] = ldg_stream2(L.blob + (size_t)(cs + (gg * (K + 1) + i) * coef_pitch));
+                        for (int i = 0; i <= K; ++i) tk.cf[q][i] = ldg_stream2(L.blob + (size_t)(cs + i * coef_pitch));
+                    }
                 } else {                              // contributes nothing: zero planes, zero coefficients
 #pragma unroll
                     for (int i = 0; i < K; ++i) tk.pl[q][i] = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                    for (int gg = 0; gg < NG; ++gg)
-#pragma unroll
-                        for (int i = 0; i <= K; ++i) tk.cf[q][gg][i] = 0;
+                    for (int i = 0; i <= K; ++i) {
+                        if constexpr (NG == 2) tk.cfp[q][i] = 0u; else tk.cf[q][i] = 0;
+                    }
                 }
             }
         };
@@ -459,28 +473,37 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                     S[NS - 1] = (e.x + e.y) + (o.x + o.y);
                 }
                 const int blk = 2 * q + h;
-                if (G64) {
-                    const float c0l = __half2float(__ushort_as_half(tk.cf[q][0][0]));
-                    const float c0h = __half2float(__ushort_as_half(tk.cf[q][NG - 1][0]));
+                if constexpr (G64) {
+                    // swap with the pair's other lane: word = (even row, odd row) of one group; this lane's row is half a & 1
+                    float cl[K + 1], ch[K + 1];       // this row's coefficients of the block's first and second group
+#pragma unroll
+                    for (int i = 0; i <= K; ++i) {
+                        const unsigned mine = tk.cfp[q][i];
+                        const unsigned other = __shfl_xor_sync(0xffffffffu, mine, 1);
+                        const unsigned g0 = (a & 1) ? other : mine, g1 = (a & 1) ? mine : other;   // words of group 0 and group 1
+                        cl[i] = __half2float(__ushort_as_half((unsigned short)((a & 1) ? (g0 >> 16) : (g0 & 0xffffu))));
+                        ch[i] = __half2float(__ushort_as_half((unsigned short)((a & 1) ? (g1 >> 16) : (g1 & 0xffffu))));
+                    }
+                    const float c0l = cl[0], c0h = ch[0];
 #pragma unroll
                     for (int m = 0; m < MT; ++m)
                         yacc[m] = fmaf(c0h, xsum[(m * kSliceBlocks + blk) * 2 + 1], fmaf(c0l, xsum[(m * kSliceBlocks + blk) * 2], yacc[m]));
 #pragma unroll
                     for (int i = 0; i < K; ++i) {
-                        const float cil = __half2float(__ushort_as_half(tk.cf[q][0][i + 1]));
-                        const float cih = __half2float(__ushort_as_half(tk.cf[q][NG - 1][i + 1]));
+                        const float cil = cl[i + 1];
+                        const float cih = ch[i + 1];
 #pragma unroll
                         for (int m = 0; m < MT; ++m)
                             yacc[m] = fmaf(cih, S[i * MT + m] - Slo[i * MT + m], fmaf(cil, Slo[i * MT + m], yacc[m]));
                     }
                 } else {
-                    const float c0 = __half2float(__ushort_as_half(tk.cf[q][0][0]));
+                    const float c0 = __half2float(__ushort_as_half(tk.cf[q][0]));
 #pragma unroll
                     for (int m = 0; m < MT; ++m)
                         yacc[m] = fmaf(c0, xsum[(m * kSliceBlocks + blk) * 2] + xsum[(m * kSliceBlocks + blk) * 2 + 1], yacc[m]);
 #pragma unroll
                     for (int i = 0; i < K; ++i) {
-                        const float ci = __half2float(__ushort_as_half(tk.cf[q][0][i + 1]));
+                        const float ci = __half2float(__ushort_as_half(tk.cf[q][i + 1]));
 #pragma unroll
                         for (int m = 0; m < MT; ++m) yacc[m] = fmaf(ci, S[i * MT + m], yacc[m]);
                     }
@@ -569,11 +592,10 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
 }
 
 // Tasks kept in flight per lane: two (a third costs more in registers than it hides in latency: measured slower
-// for every K); one where two tasks do not fit the register file (K = 4; K >= 3 with the second coefficient
-// group of g = 64).
+// for every K); one where two tasks do not fit the register file (K = 4).
 template <int K, int MT>
 int launch_one(bpdq_handle_s* h, const GemvParams& p, cudaStream_t stream) {
-    if (p.lin[0].group == 64) return launch_cfg<K, MT, (K <= 2 ? 2 : 1), 16, true>(h, p, stream);
+    if (p.lin[0].group == 64) return launch_cfg<K, MT, (K <= 3 ? 2 : 1), 16, true>(h, p, stream);
     return launch_cfg<K, MT, (K <= 3 ? 2 : 1), 16, false>(h, p, stream);
 }
 
