@@ -40,7 +40,7 @@ HBM_NOMINAL_GBS = 8000.0
 FALLBACK_HBM_GBS, FALLBACK_TFLOPS = 6650.0, 1590.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the headline launch, from one ncu capture of this kernel as it stands
 # (set to None whenever the kernel changes until the counters are taken again)
-GEMV_TRAFFIC_BYTES_PER_LAUNCH = 264_921_088
+GEMV_TRAFFIC_BYTES_PER_LAUNCH = 267_311_616
 
 
 def useful_bytes(out: int, in_: int, K: int, g: int, M: int) -> int:
