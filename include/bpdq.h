@@ -26,6 +26,11 @@
  *     that take a stream only enqueue work and do not synchronise, unless stated;
  *   - a handle owns its device copy of the packed weights and a scratch workspace.  Two calls
  *     on the same handle must not overlap on the GPU (issue them on one stream);
+ *   - threads: calls that name the same handle (for bpdq_linear_batch: the same first handle,
+ *     which keeps the launch plan) and all calls of bpdq_linear_noalloc on one device must be
+ *     serialised by the caller; calls on different handles may run concurrently from
+ *     different threads.  A handle is used with the device that was current when it was
+ *     created: calling with another current device is BPDQ_ERR_INVALID, nothing is launched;
  *   - supported shapes: K in {1,2,3,4}; g in {64,128,256}; in % 128 == 0 and in % g == 0;
  *     out % 16 == 0.  Anything else is BPDQ_ERR_UNSUPPORTED.
  *
@@ -181,7 +186,9 @@ BPDQ_API int bpdq_linear_host(bpdq_handle_t h, const void* x_fp16_host, void* y_
  * make that first call outside any stream capture.  No call allocates or frees device or host
  * memory.  Every call on a device uses the same array: it is cleared on `stream` before the
  * kernel runs, so two calls that overlap on the GPU (different streams, different threads)
- * race on it -- issue them on one stream.  Asynchronous like bpdq_linear. */
+ * race on it -- issue them on one stream.  Asynchronous like bpdq_linear.  There is no handle, so
+ * bpdq_get_status cannot report on these calls: the status word lives in the same array and is
+ * cleared by the next call. */
 BPDQ_API int bpdq_linear_noalloc(const void* blob_dev, int out, int in, int K, int group, const void* x_fp16_dev,
                         void* y_fp16_dev, int M, void* stream);
 

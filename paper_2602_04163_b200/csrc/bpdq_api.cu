@@ -58,12 +58,44 @@ void* mapped_address(const void* host) {
     return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
 }
 
+// A handle's buffers live on the device that was current in bpdq_create; a launch under another current device
+// would hand that device pointers it cannot use.
+int check_device(const bpdq_handle_s* h, const char* who) {
+    int dev = -1;
+    const cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return set_error(BPDQ_ERR_CUDA, "%s: cudaGetDevice: %s", who, cudaGetErrorString(e));
+    if (dev != h->device)
+        return set_error(BPDQ_ERR_INVALID, "%s: the handle lives on device %d, the current device is %d", who, h->device, dev);
+    return BPDQ_OK;
+}
+
 int check_linear_args(bpdq_handle_s* h, const void* x, void* y, int M, const char* who) {
     if (!h) return set_error(BPDQ_ERR_INVALID, "%s: null handle", who);
     if (M < 0 || M > h->max_M) return set_error(BPDQ_ERR_INVALID, "%s: M=%d outside [0, max_M=%d]", who, M, h->max_M);
     if (M == 0) return BPDQ_OK;
     if (!x || !y) return set_error(BPDQ_ERR_INVALID, "%s: null pointer", who);
-    return BPDQ_OK;
+    return check_device(h, who);
+}
+
+// Everything bpdq_linear_batch requires of its handles and of M (pointers are checked by the callers, which
+// differ in where those pointers live).
+int check_batch_handles(const bpdq_handle_t* hs, int n, int M, const char* who) {
+    if (!hs) return set_error(BPDQ_ERR_INVALID, "%s: null array", who);
+    if (n < 1 || n > BPDQ_BATCH_MAX) return set_error(BPDQ_ERR_INVALID, "%s: n=%d outside [1, %d]", who, n, BPDQ_BATCH_MAX);
+    if (M < 0 || M > BPDQ_GEMV_MAX_M) return set_error(BPDQ_ERR_INVALID, "%s: M=%d outside [0, %d]", who, M, BPDQ_GEMV_MAX_M);
+    for (int k = 0; k < n; ++k) {
+        if (!hs[k]) return set_error(BPDQ_ERR_INVALID, "%s: null handle at %d", who, k);
+        if (M > hs[k]->max_M) return set_error(BPDQ_ERR_INVALID, "%s: M=%d exceeds max_M=%d of linear %d", who, M, hs[k]->max_M, k);
+        if (hs[k]->K != hs[0]->K || hs[k]->device != hs[0]->device)
+            return set_error(BPDQ_ERR_INVALID, "%s: linear %d differs from linear 0 in K or device", who, k);
+        if ((hs[k]->group == 64) != (hs[0]->group == 64))
+            return set_error(BPDQ_ERR_INVALID, "%s: linear %d and linear 0 differ in having group 64", who, k);
+        if (!gemv_supported(hs[k]->out, hs[k]->in, hs[k]->K, hs[k]->group))
+            return set_error(BPDQ_ERR_UNSUPPORTED, "%s: look-up-table kernel does not cover linear %d (K=%d g=%d; packed weights must stay below 4 GB)", who, k, hs[k]->K, hs[k]->group);
+        for (int j = 0; j < k; ++j)
+            if (hs[j] == hs[k]) return set_error(BPDQ_ERR_INVALID, "%s: handle %d repeats handle %d", who, k, j);
+    }
+    return M == 0 ? BPDQ_OK : check_device(hs[0], who);
 }
 
 }  // namespace
@@ -141,6 +173,7 @@ extern "C" int bpdq_dequant(bpdq_handle_t h, void* w, void* stream) {
     if (!h) return set_error(BPDQ_ERR_INVALID, "bpdq_dequant: null handle");
     if (!w) return set_error(BPDQ_ERR_INVALID, "bpdq_dequant: null output pointer");
     if (!aligned16(w)) return set_error(BPDQ_ERR_INVALID, "bpdq_dequant: output pointer not 16-byte aligned");
+    if (const int rc = check_device(h, "bpdq_dequant"); rc != BPDQ_OK) return rc;
     return launch_dequant(h, w, static_cast<cudaStream_t>(stream));
 }
 
@@ -177,23 +210,11 @@ extern "C" int bpdq_linear_ex(bpdq_handle_t h, const void* x, void* y, int M, in
 
 extern "C" int bpdq_linear_batch(const bpdq_handle_t* hs, const void* const* xs, void* const* ys, int n, int M, void* stream) {
     if (!hs || !xs || !ys) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: null array");
-    if (n < 1 || n > BPDQ_BATCH_MAX) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: n=%d outside [1, %d]", n, BPDQ_BATCH_MAX);
-    if (M < 0 || M > BPDQ_GEMV_MAX_M) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: M=%d outside [0, %d]", M, BPDQ_GEMV_MAX_M);
-    for (int k = 0; k < n; ++k) {
-        if (!hs[k]) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: null handle at %d", k);
-        if (M > hs[k]->max_M) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: M=%d exceeds max_M=%d of linear %d", M, hs[k]->max_M, k);
-        if (hs[k]->K != hs[0]->K || hs[k]->device != hs[0]->device)
-            return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: linear %d differs from linear 0 in K or device", k);
-        if ((hs[k]->group == 64) != (hs[0]->group == 64))
-            return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: linear %d and linear 0 differ in having group 64", k);
-        if (!gemv_supported(hs[k]->out, hs[k]->in, hs[k]->K, hs[k]->group))
-            return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear_batch: look-up-table kernel does not cover linear %d (K=%d g=%d; packed weights must stay below 4 GB)", k, hs[k]->K, hs[k]->group);
-        for (int j = 0; j < k; ++j)
-            if (hs[j] == hs[k]) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: handle %d repeats handle %d", k, j);
-        if (M > 0 && (!xs[k] || !ys[k] || !aligned16(xs[k]) || !aligned16(ys[k])))
-            return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: x and y of linear %d must be non-null and 16-byte aligned", k);
-    }
+    if (const int rc = check_batch_handles(hs, n, M, "bpdq_linear_batch"); rc != BPDQ_OK) return rc;
     if (M == 0) return BPDQ_OK;
+    for (int k = 0; k < n; ++k)
+        if (!xs[k] || !ys[k] || !aligned16(xs[k]) || !aligned16(ys[k]))
+            return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: x and y of linear %d must be non-null and 16-byte aligned", k);
     return launch_gemv_batch(hs, xs, ys, n, M, static_cast<cudaStream_t>(stream));
 }
 
@@ -221,13 +242,11 @@ extern "C" int bpdq_linear_host(bpdq_handle_t h, const void* x_host, void* y_hos
 extern "C" int bpdq_linear_batch_host(const bpdq_handle_t* hs, const void* const* xs_host, void* const* ys_host, int n, int M,
                                       void* stream) {
     if (!hs || !xs_host || !ys_host) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch_host: null array");
-    if (n < 1 || n > BPDQ_BATCH_MAX) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch_host: n=%d outside [1, %d]", n, BPDQ_BATCH_MAX);
-    for (int k = 0; k < n; ++k) {
-        if (!hs[k]) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch_host: null handle at %d", k);
-        if (M < 0 || M > hs[k]->max_M) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch_host: M=%d outside [0, max_M=%d] of linear %d", M, hs[k]->max_M, k);
-        if (M > 0 && (!xs_host[k] || !ys_host[k])) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch_host: null pointer at %d", k);
-    }
+    // every rule of bpdq_linear_batch is checked before anything is enqueued
+    if (const int rc = check_batch_handles(hs, n, M, "bpdq_linear_batch_host"); rc != BPDQ_OK) return rc;
     if (M == 0) return BPDQ_OK;
+    for (int k = 0; k < n; ++k)
+        if (!xs_host[k] || !ys_host[k]) return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch_host: null pointer at %d", k);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const void* xd[BPDQ_BATCH_MAX];
     void* yd[BPDQ_BATCH_MAX];
@@ -255,9 +274,9 @@ extern "C" int bpdq_linear_batch_host(const bpdq_handle_t* hs, const void* const
             unsigned blocks = (end16 + 1023u) / 1024u;
             if (blocks > 64u) blocks = 64u;
             gather_kernel<<<blocks, 1024, 0, s>>>(g);
-            hs[0]->launches += 1;
             cudaError_t e = cudaGetLastError();
             if (e != cudaSuccess) return cuda_fail("bpdq_linear_batch_host: gather launch", e);
+            hs[0]->launches += 1;
             const int rc = bpdq_linear_batch(hs, xd, yd, n, M, stream);
             if (rc != BPDQ_OK) return rc;
             e = cudaStreamSynchronize(s);
@@ -292,6 +311,7 @@ extern "C" int bpdq_set_gemv_max_m(bpdq_handle_t h, int max_gemv_m) {
 
 extern "C" int bpdq_read_blob(bpdq_handle_t h, void* host_blob) {
     if (!h || !host_blob) return set_error(BPDQ_ERR_INVALID, "bpdq_read_blob: null pointer");
+    if (const int rc = check_device(h, "bpdq_read_blob"); rc != BPDQ_OK) return rc;
     cudaError_t e = cudaMemcpy(host_blob, h->d_blob, h->blob_bytes, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail("bpdq_read_blob", e);
     return BPDQ_OK;
@@ -299,6 +319,7 @@ extern "C" int bpdq_read_blob(bpdq_handle_t h, void* host_blob) {
 
 extern "C" int bpdq_get_status(bpdq_handle_t h, void* stream) {
     if (!h) return set_error(BPDQ_ERR_INVALID, "bpdq_get_status: null handle");
+    if (const int rc = check_device(h, "bpdq_get_status"); rc != BPDQ_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int st = 0;
     cudaError_t e = cudaMemcpyAsync(&st, h->d_status, sizeof(int), cudaMemcpyDeviceToHost, s);

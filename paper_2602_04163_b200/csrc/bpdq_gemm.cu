@@ -699,12 +699,8 @@ EncodeTiledFn encode_tiled_fn() {
 template <int K, int BN>
 int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
     using C = TileCfg<K, BN>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<K, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-        if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: shared memory opt-in: %s", cudaGetErrorString(e));
-        configured = true;
-    }
+    static bpdq::SmemOptin optin;
+    if (const int rc = bpdq::ensure_smem_optin(gemm_kernel<K, BN>, optin, h->device, C::kSmemBytes, "gemm"); rc != BPDQ_OK) return rc;
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: cuTensorMapEncodeTiled is not available from this driver");
     CUtensorMap map;
@@ -765,12 +761,8 @@ int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t st
 template <int K>
 int launch_persistent(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
     using C = Cfg<K, kPersistBN>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_persistent_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-        if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: shared memory opt-in: %s", cudaGetErrorString(e));
-        configured = true;
-    }
+    static bpdq::SmemOptin optin;
+    if (const int rc = bpdq::ensure_smem_optin(gemm_persistent_kernel<K>, optin, h->device, C::kSmemBytes, "gemm"); rc != BPDQ_OK) return rc;
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: cuTensorMapEncodeTiled is not available from this driver");
     CUtensorMap map;

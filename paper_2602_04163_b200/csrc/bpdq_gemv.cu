@@ -88,10 +88,12 @@ __device__ __forceinline__ uint4 ldg_stream16(const uint8_t* p) {
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
-// volatile, so that it stays ahead of the weight requests issued after it
-__device__ __forceinline__ unsigned ldg_first4(const void* p) {
+// Activations: the kernel before this one in the stream may have written them while this kernel was already
+// resident, so they are read through the coherent path (L2), never the read-only one.  Volatile, so that the
+// load stays behind griddepcontrol.wait and ahead of the weight requests issued after it.
+__device__ __forceinline__ unsigned ldg_x4(const void* p) {
     unsigned v;
-    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
 __device__ __forceinline__ unsigned ldg_stream4(const uint8_t* p) {
@@ -348,7 +350,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
         for (int m = 0; m < MT; ++m)
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                xraw[m][u] = col < L.in ? ldg_first4(L.x + (size_t)m * L.in + col + 8 * u) : 0u;
+                xraw[m][u] = col < L.in ? ldg_x4(L.x + (size_t)m * L.in + col + 8 * u) : 0u;
         if (!early) {
 #pragma unroll
             for (int d = 0; d < D; ++d)
@@ -540,15 +542,11 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
 
 template <int K, int MT, int D, int W, bool G64>
 int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
-    static int configured_smem = 0;
+    static bpdq::SmemOptin optin;
     const int smem = 65536 + MT * kTableBytes;        // tables start at the first 64 KB boundary of the shared window
     if (smem > h->smem_optin)
         return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv: %d bytes of shared memory needed, device offers %d", smem, h->smem_optin);
-    if (configured_smem != smem) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_lut_kernel<K, MT, D, W, G64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemv: shared memory opt-in: %s", cudaGetErrorString(e));
-        configured_smem = smem;
-    }
+    if (const int rc = bpdq::ensure_smem_optin(gemv_lut_kernel<K, MT, D, W, G64>, optin, h->device, smem, "gemv"); rc != BPDQ_OK) return rc;
     long long total = 0;
     for (int k = 0; k < p.n; ++k) {
         if ((unsigned long long)p.lin[k].blob_bytes >= (1ull << 32))
@@ -692,11 +690,12 @@ constexpr size_t kNoallocBytes = kNoallocWsBytes + kNoallocCounterBytes + 256;  
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoallocBytes];
 
-constexpr int kMaxDevices = 64;
+using bpdq::kMaxDevices;
 struct NoallocDevice {
     bool ready;
     unsigned char* scratch;       // device address of g_noalloc_scratch on this device
     int sm_count, smem_optin;
+    bpdq_handle_s view;           // what the launcher sees; owns nothing, keeps the last cut of the task space between calls
 };
 NoallocDevice g_noalloc_dev[kMaxDevices];
 
@@ -741,7 +740,7 @@ extern "C" int bpdq_linear_noalloc(const void* blob_dev, int out, int in, int K,
     if (dev < 0 || dev >= kMaxDevices) return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear_noalloc: device ordinal %d", dev);
     int rc = noalloc_setup(dev);
     if (rc != BPDQ_OK) return rc;
-    const NoallocDevice& d = g_noalloc_dev[dev];
+    NoallocDevice& d = g_noalloc_dev[dev];
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
     // The scratch keeps whatever the last call left; the kernel needs row sums and counters at zero.
@@ -750,7 +749,7 @@ extern "C" int bpdq_linear_noalloc(const void* blob_dev, int out, int in, int K,
         (e = cudaMemsetAsync(d.scratch + kNoallocWsBytes, 0, kNoallocCounterBytes + 256, s)) != cudaSuccess)
         return set_error(BPDQ_ERR_CUDA, "bpdq_linear_noalloc: clearing the scratch: %s", cudaGetErrorString(e));
 
-    bpdq_handle_s h{};                                   // a view for the launcher; owns nothing
+    bpdq_handle_s& h = d.view;                          // calls with the shape of the last one reuse its cut (launch_cfg compares shapes)
     h.out = out; h.in = in; h.K = K; h.group = group; h.max_M = BPDQ_GEMV_MAX_M; h.device = dev;
     h.sm_count = d.sm_count; h.smem_optin = d.smem_optin;
     h.d_blob = const_cast<uint8_t*>(static_cast<const uint8_t*>(blob_dev));

@@ -33,6 +33,23 @@ BPDQ_HD size_t coefs_bytes(int64_t out, int64_t in, int K, int64_t g) {
 bool shape_supported(int out, int in, int K, int group);
 int set_error(int code, const char* fmt, ...);
 
+// Opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of a kernel: one record per kernel
+// instantiation, indexed by device ordinal.  Setting the attribute twice is harmless, so concurrent first calls
+// need no lock; the record only saves the runtime call on later launches.
+constexpr int kMaxDevices = 64;
+struct SmemOptin {
+    int bytes[kMaxDevices];       // largest size opted in to on each device so far (zero-initialised as a static)
+};
+template <typename Kernel>
+inline int ensure_smem_optin(Kernel kernel, SmemOptin& rec, int device, int bytes, const char* who) {
+    if (device < 0 || device >= kMaxDevices) return set_error(BPDQ_ERR_UNSUPPORTED, "%s: device ordinal %d", who, device);
+    if (__atomic_load_n(&rec.bytes[device], __ATOMIC_ACQUIRE) >= bytes) return BPDQ_OK;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return set_error(BPDQ_ERR_CUDA, "%s: shared memory opt-in: %s", who, cudaGetErrorString(e));
+    __atomic_store_n(&rec.bytes[device], bytes, __ATOMIC_RELEASE);
+    return BPDQ_OK;
+}
+
 }  // namespace bpdq
 
 struct bpdq_handle_s {

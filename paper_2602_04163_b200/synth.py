@@ -130,9 +130,10 @@ def coefficients(seed: int, out: int, in_: int, K: int, group: int, rows=None) -
     return res
 
 
-def activations(seed: int, M: int, in_: int) -> np.ndarray:
-    """fp16 bit patterns of x, uint16 [M][in]."""
-    e = np.arange(M * in_, dtype=np.uint64).reshape(M, in_)
+def activations(seed: int, M: int, in_: int, tokens=None) -> np.ndarray:
+    """fp16 bit patterns of x, uint16 [M][in]; with `tokens` only those token rows, uint16 [len(tokens)][in]."""
+    t = _rows(M, tokens)
+    e = t[:, None] * np.uint64(in_) + np.arange(in_, dtype=np.uint64)[None, :]
     v = _irwin_hall_int(seed, TENSOR_X, e).astype(np.float32) * X_SCALE
     return v.astype(np.float16).view(np.uint16)
 

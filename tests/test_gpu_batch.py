@@ -53,6 +53,22 @@ def test_batch_rejects_bad_arguments():
     binding.bpdq_linear_batch([h1], [0], [0], 0, G.stream_ptr())              # M = 0: nothing to do
 
 
+def test_batch_host_rejects_before_anything_is_enqueued():
+    """The host-buffer call checks every rule of bpdq_linear_batch first: a rejected call launches nothing
+    (not even the kernel that gathers the inputs)."""
+    h1, _, _ = G.make_layer(1, 32, 128, 2, 128, max_M=2)
+    h2, _, _ = G.make_layer(2, 32, 128, 3, 128, max_M=2)
+    xh = torch.zeros((2, 128), dtype=torch.float16).pin_memory()
+    yh = [torch.zeros((2, 32), dtype=torch.float16).pin_memory() for _ in range(2)]
+    n0 = h1.bpdq_launch_count() + h2.bpdq_launch_count()
+    for handles, M in (([h1, h1], 1), ([h1, h2], 1), ([h1], 3), ([h1], binding.GEMV_MAX_M + 1)):
+        with pytest.raises(binding.BpdqError) as ei:
+            binding.bpdq_linear_batch_host(handles, [xh.data_ptr()] * len(handles), [y.data_ptr() for y in yh][:len(handles)], M,
+                                           G.stream_ptr())
+        assert ei.value.code == binding.ERR_INVALID
+    assert h1.bpdq_launch_count() + h2.bpdq_launch_count() == n0
+
+
 @pytest.mark.parametrize("model,K", [("72b", 2), ("72b", 3), ("7b", 2)])
 def test_batch_full_layer_sampled(model, K):
     """All seven linears of a Qwen2.5-shaped layer in one launch (the benchmark's step); sampled rows against the checker."""
@@ -71,7 +87,8 @@ def test_batch_full_layer_sampled(model, K):
         h.bpdq_destroy()
 
 
-@pytest.mark.parametrize("name,out,in_,K", [("gate", 29568, 8192, 2), ("down", 8192, 29568, 3)])
+@pytest.mark.parametrize("name,out,in_,K", [("gate", 29568, 8192, 2), ("gate", 29568, 8192, 3), ("down", 8192, 29568, 2),
+                                             ("down", 8192, 29568, 3)])
 def test_token_sweep_through_the_dispatcher(name, out, in_, K):
     """M = 1..64 on 72B-shaped projections through bpdq_linear (look-up-table kernel below the threshold,
     tensor-core kernel above); sampled rows against the checker."""

@@ -14,7 +14,8 @@ from tests import gpu_util as G
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("K,g,out,in_,M", [(2, 128, 4096, 4096, 1), (3, 128, 272, 896, 3), (2, 256, 64, 1024, 2)])
+@pytest.mark.parametrize("K,g,out,in_,M", [(2, 128, 4096, 4096, 1), (3, 128, 272, 896, 3), (2, 256, 64, 1024, 2),
+                                            (1, 128, 65536, 128, 3)])     # the most rows it takes: last counter, last scratch row, two passes
 def test_noalloc_matches_handle_kernel_twice(K, g, out, in_, M):
     import torch
     h, bits, coef = G.make_layer(80 + K, out, in_, K, g, max_M=M)
