@@ -1,6 +1,7 @@
 """Benchmark of the BPDQ weight-only linear layer (decode GEMV, prefill GEMM, dequant) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-extras]
+    python bench.py --case few --out 29568 --in 8192 --K 2 --M 16 --iters 3      (one kernel on one linear, for profilers)
 
 One JSON line on stdout.  The headline workload is a Qwen2.5-72B-shaped decoder layer at K = 2
 bit-planes, group 128, one token (M = 1): a step is one pass of bpdq_linear over the layer's seven
@@ -560,6 +561,54 @@ def full_stack_section(torch, binding, peaks, sp, stream, n_layers=80):
     return res
 
 
+def run_case(a):
+    """One kernel of the library a few times on one synthetic linear (or the 72B-shaped layer in one batched launch):
+    the small, single-kernel command that profiler captures are taken from.  Prints the median launch time."""
+    import torch
+    from paper_2602_04163_b200 import binding
+    kernels = {"auto": binding.KERNEL_AUTO, "gemv": binding.KERNEL_GEMV, "gemm": binding.KERNEL_GEMM,
+               "simple": binding.KERNEL_GEMV_SIMPLE, "few": binding.KERNEL_FEW}
+    torch.cuda.set_device(0)
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if a.flush_l2 else None
+    M = max(1, a.M)
+    if a.case == "layer72b":
+        shapes = synth.QWEN25_72B_LAYER
+        hs = [binding.Handle(o, i, a.K, a.group, None, a.seed + li, M) for li, (_, o, i) in enumerate(shapes)]
+        xs = {i: torch.from_numpy(synth.activations(a.seed + 9, M, i).view(np.int16).copy()).cuda().view(torch.float16)
+              for i in sorted({i for _, _, i in shapes})}
+        ys = [torch.empty((M, o), dtype=torch.float16, device="cuda") for _, o, _ in shapes]
+
+        def call():
+            binding.bpdq_linear_batch(hs, [xs[h.in_].data_ptr() for h in hs], [y.data_ptr() for y in ys], M, sp)
+        what = f"layer72b batch K={a.K} g={a.group} M={M}"
+    else:
+        hs = [binding.Handle(a.out, a.in_, a.K, a.group, None, a.seed, M)]
+        x = torch.from_numpy(synth.activations(a.seed + 1, M, a.in_).view(np.int16).copy()).cuda().view(torch.float16)
+        y = torch.empty((M, a.out), dtype=torch.float16, device="cuda")
+        w = torch.empty((a.out, a.in_), dtype=torch.float16, device="cuda") if a.case == "dequant" else None
+
+        def call():
+            if a.case == "dequant":
+                hs[0].bpdq_dequant(w.data_ptr(), sp)
+            else:
+                hs[0].bpdq_linear_ex(x.data_ptr(), y.data_ptr(), M, kernels[a.case], sp)
+        what = f"{a.case} out={a.out} in={a.in_} K={a.K} g={a.group} M={M}"
+    times = []
+    for _ in range(a.iters):
+        if flush is not None:
+            flush.zero_()
+        times.append(event_time_ms(torch, call, stream))
+    hs[0].bpdq_get_status(sp)
+    times.sort()
+    med = times[len(times) // 2]
+    packed = sum(h.packed_bytes for h in hs)
+    print(f"{what}: median {med * 1e3:.1f} us over {a.iters} launches; packed {packed / 1e6:.1f} MB -> {packed / med / 1e6:.0f} GB/s")
+    for h in hs:
+        h.bpdq_destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -567,7 +616,20 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--case", default=None, choices=["auto", "gemv", "few", "gemm", "simple", "dequant", "layer72b"],
+                    help="run one kernel on one linear instead of the benchmark (for profilers)")
+    ap.add_argument("--out", type=int, default=29568)
+    ap.add_argument("--in", dest="in_", type=int, default=8192)
+    ap.add_argument("--K", type=int, default=2)
+    ap.add_argument("--group", type=int, default=128)
+    ap.add_argument("--M", type=int, default=1)
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--flush-l2", action="store_true", help="with --case: write 256 MB between launches")
     args = ap.parse_args()
+    if args.case:
+        run_case(args)
+        return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

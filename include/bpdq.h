@@ -88,10 +88,13 @@ enum {
     BPDQ_KERNEL_AUTO = 0,     /* dispatch on M (what bpdq_linear does)                        */
     BPDQ_KERNEL_GEMV = 1,     /* look-up-table kernel, M <= BPDQ_GEMV_MAX_M                   */
     BPDQ_KERNEL_GEMM = 2,     /* tensor-core kernel (TMA + tcgen05), any M >= 1               */
-    BPDQ_KERNEL_GEMV_SIMPLE = 3 /* one-bit-at-a-time kernel kept as an on-device cross-check  */
+    BPDQ_KERNEL_GEMV_SIMPLE = 3, /* one-bit-at-a-time kernel kept as an on-device cross-check */
+    BPDQ_KERNEL_FEW = 4       /* few-token kernel (weights decoded in registers, warp-level
+                                 tensor-core instructions), M <= BPDQ_FEW_MAX_M              */
 };
 
 #define BPDQ_GEMV_MAX_M 16
+#define BPDQ_FEW_MAX_M 32
 #define BPDQ_BATCH_MAX 16            /* most linears bpdq_linear_batch takes in one call */
 #define BPDQ_NOALLOC_MAX_OUT 65536   /* most output rows bpdq_linear_noalloc accepts */
 
@@ -126,10 +129,10 @@ BPDQ_API int bpdq_dequant(bpdq_handle_t h, void* w_fp16_dev, void* stream);
 
 /* The quantized linear map y = x * W^T (paper: Eq. 1 applied to activations, Section 3.1).
  * x: device binary16 [M][in]; y: device binary16 [M][out]; 0 <= M <= max_M.  M == 0 returns
- * BPDQ_OK without a launch.  Picks the look-up-table kernel for small M and the tensor-core
- * kernel above the handle's dispatch threshold (and for every M when the packed weights of the
- * linear reach 4 GB, which the look-up-table kernel's 32-bit offsets do not cover).  x and y must
- * not alias. */
+ * BPDQ_OK without a launch.  Picks the look-up-table kernel for the smallest M (default: up to
+ * 2 tokens), the few-token kernel above that (default: up to 16 tokens) and the tcgen05 kernel
+ * beyond (also below when the packed weights of the linear reach 4 GB, which the look-up-table
+ * kernel's 32-bit offsets do not cover).  x and y must not alias. */
 BPDQ_API int bpdq_linear(bpdq_handle_t h, const void* x_fp16_dev, void* y_fp16_dev, int M, void* stream);
 
 /* Same map with the kernel chosen by the caller (BPDQ_KERNEL_*).  BPDQ_KERNEL_GEMV with
@@ -137,11 +140,12 @@ BPDQ_API int bpdq_linear(bpdq_handle_t h, const void* x_fp16_dev, void* y_fp16_d
 BPDQ_API int bpdq_linear_ex(bpdq_handle_t h, const void* x_fp16_dev, void* y_fp16_dev, int M, int kernel,
                    void* stream);
 
-/* Several independent linears in one launch of the look-up-table kernel (decode: q, k, v of one
- * token, or gate and up, or a whole layer's linears when their inputs do not depend on each
- * other).  y[k] = x[k] * W^[k]^T for k = 0..n-1, each exactly as bpdq_linear with
- * BPDQ_KERNEL_GEMV computes it; the task spaces of the n linears are concatenated, so launch
- * ramp, table set-up and tail are paid once instead of n times.  hs, xs, ys are HOST arrays of n
+/* Several independent linears in one launch (decode: q, k, v of one token, or gate and up, or a
+ * whole layer's linears when their inputs do not depend on each other).  y[k] = x[k] * W^[k]^T
+ * for k = 0..n-1, each as bpdq_linear computes it for this M: the look-up-table kernel up to the
+ * first handle's look-up-table threshold, the few-token kernel above it (up to its threshold,
+ * when every linear allows it), else passes of the look-up-table kernel; the task spaces of the
+ * n linears are concatenated, so launch ramp, set-up and tail are paid once instead of n times.  hs, xs, ys are HOST arrays of n
  * handles / device pointers (read before the call returns); 1 <= n <= BPDQ_BATCH_MAX; the
  * handles are distinct, live on the current device, share K, and either all or none of them
  * have group 64;
@@ -195,6 +199,10 @@ BPDQ_API int bpdq_linear_noalloc(const void* blob_dev, int out, int in, int K, i
 /* Sets the largest M that bpdq_linear sends to the look-up-table kernel (0 = always use the
  * tensor-core kernel; at most BPDQ_GEMV_MAX_M). */
 BPDQ_API int bpdq_set_gemv_max_m(bpdq_handle_t h, int max_gemv_m);
+
+/* Sets the largest M that bpdq_linear sends to the few-token kernel once M is above the look-up-table
+ * threshold (0 = never; at most BPDQ_FEW_MAX_M and the handle's max_M). */
+BPDQ_API int bpdq_set_few_max_m(bpdq_handle_t h, int max_few_m);
 
 /* Copies the device blob back to host memory (bpdq_packed_bytes() bytes); synchronises. */
 BPDQ_API int bpdq_read_blob(bpdq_handle_t h, void* host_blob);

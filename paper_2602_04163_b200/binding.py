@@ -16,12 +16,13 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libbpdq.so")
 
 OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(6)
-KERNEL_AUTO, KERNEL_GEMV, KERNEL_GEMM, KERNEL_GEMV_SIMPLE = range(4)
+KERNEL_AUTO, KERNEL_GEMV, KERNEL_GEMM, KERNEL_GEMV_SIMPLE, KERNEL_FEW = range(5)
 GEMV_MAX_M = 16
+FEW_MAX_M = 32
 NOALLOC_MAX_OUT = 65536
 
 EXPORTS = ("bpdq_packed_bytes", "bpdq_pack", "bpdq_unpack", "bpdq_create", "bpdq_dequant", "bpdq_linear",
-           "bpdq_linear_ex", "bpdq_linear_host", "bpdq_set_gemv_max_m", "bpdq_read_blob", "bpdq_get_status",
+           "bpdq_linear_ex", "bpdq_linear_host", "bpdq_set_gemv_max_m", "bpdq_set_few_max_m", "bpdq_read_blob", "bpdq_get_status",
            "bpdq_launch_count", "bpdq_destroy", "bpdq_last_error", "bpdq_linear_noalloc", "bpdq_linear_batch", "bpdq_linear_batch_host")
 
 _lib = None
@@ -55,6 +56,7 @@ def lib() -> ctypes.CDLL:
         L.bpdq_linear_batch_host.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), i, i, vp]
         L.bpdq_linear_noalloc.argtypes = [vp, i, i, i, i, vp, vp, i, vp]
         L.bpdq_set_gemv_max_m.argtypes = [vp, i]
+        L.bpdq_set_few_max_m.argtypes = [vp, i]
         L.bpdq_read_blob.argtypes = [vp, vp]
         L.bpdq_get_status.argtypes = [vp, vp]
         L.bpdq_launch_count.argtypes = [vp, ctypes.POINTER(u64)]
@@ -167,6 +169,9 @@ class Handle:
 
     def bpdq_set_gemv_max_m(self, m: int) -> None:
         _check(lib().bpdq_set_gemv_max_m(self._h, m))
+
+    def bpdq_set_few_max_m(self, m: int) -> None:
+        _check(lib().bpdq_set_few_max_m(self._h, m))
 
     def bpdq_read_blob(self) -> np.ndarray:
         blob = np.empty(self.packed_bytes, dtype=np.uint8)

@@ -24,6 +24,7 @@ void free_handle(bpdq_handle_s* h) {
     if (h->d_status) cudaFree(h->d_status);
     if (h->d_xstage) cudaFree(h->d_xstage);
     if (h->d_ystage) cudaFree(h->d_ystage);
+    if (h->d_few_maps) cudaFree(h->d_few_maps);
     delete h;
 }
 
@@ -127,9 +128,13 @@ extern "C" int bpdq_create(bpdq_handle_t* hp, int out, int in, int K, int group,
     h->blob_bytes = h->planes_bytes + coefs_bytes(out, in, K, group);
     h->ws_bytes = gemv_workspace_bytes(out, in, K, group, max_M, h->sm_count);
     h->n_counters = gemv_counter_count(out);
-    // Measured crossover on 72B-shaped layers: two two-token passes of the look-up-table kernel (about 75 us on
-    // the largest projections) still beat the tensor-core kernel (86-94 us up to 64 tokens), a third pass does not.
-    h->gemv_max_m = 4;
+    // Measured on 72B-shaped layers: one two-token pass of the look-up-table kernel (37 us on the largest projections)
+    // beats every other kernel; a second pass (64 us) does not beat the few-token kernel.
+    h->gemv_max_m = 2;
+    // 3 to 16 tokens: the few-token kernel reads the weights once (45-60 us on the largest 72B-shaped projections
+    // against 64 us for two look-up-table passes and 67-75 us for the tcgen05 tile kernel); from 17 tokens on its second
+    // token tile costs more than the tile kernel.
+    h->few_max_m = 16;
 
     const size_t stage_x = (size_t)max_M * in * 2, stage_y = (size_t)max_M * out * 2;
     if ((e = cudaMalloc(&h->d_blob, h->blob_bytes)) != cudaSuccess ||
@@ -145,7 +150,8 @@ extern "C" int bpdq_create(bpdq_handle_t* hp, int out, int in, int K, int group,
     cudaMemset(h->d_counters, 0, (h->n_counters ? h->n_counters : 1) * sizeof(unsigned));
     cudaMemset(h->d_status, 0, sizeof(int));
     cudaMemset(h->d_ws, 0, h->ws_bytes ? h->ws_bytes : 16);
-    int rc = BPDQ_OK;
+    int rc = few_prepare(h);
+    if (rc != BPDQ_OK) { free_handle(h); return rc; }
     if (host_blob) {
         e = cudaMemcpy(h->d_blob, host_blob, h->blob_bytes, cudaMemcpyHostToDevice);
         if (e != cudaSuccess) rc = cuda_fail("bpdq_create: blob copy", e);
@@ -186,7 +192,9 @@ extern "C" int bpdq_linear_ex(bpdq_handle_t h, const void* x, void* y, int M, in
     if (kernel == BPDQ_KERNEL_AUTO) {
         const bool gv = gemv_supported(h->out, h->in, h->K, h->group);
         const bool gm = gemm_supported(h->out, h->in, h->K, h->group);
+        const bool fw = gemv_mma_supported(h->out, h->in, h->K, h->group);
         if (gv && (M <= h->gemv_max_m || !gm) && M <= BPDQ_GEMV_MAX_M) kernel = BPDQ_KERNEL_GEMV;
+        else if (fw && M <= h->few_max_m && M <= BPDQ_FEW_MAX_M) kernel = BPDQ_KERNEL_FEW;
         else if (gm) kernel = BPDQ_KERNEL_GEMM;
         else kernel = BPDQ_KERNEL_GEMV_SIMPLE;
     }
@@ -203,6 +211,12 @@ extern "C" int bpdq_linear_ex(bpdq_handle_t h, const void* x, void* y, int M, in
             return launch_gemm(h, x, y, M, s);
         case BPDQ_KERNEL_GEMV_SIMPLE:
             return launch_gemv_simple(h, x, y, M, s);
+        case BPDQ_KERNEL_FEW:
+            if (M > BPDQ_FEW_MAX_M)
+                return set_error(BPDQ_ERR_INVALID, "bpdq_linear: few-token kernel takes M <= %d, got %d", BPDQ_FEW_MAX_M, M);
+            if (!gemv_mma_supported(h->out, h->in, h->K, h->group))
+                return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_linear: few-token kernel does not cover this linear (K=%d g=%d)", h->K, h->group);
+            return launch_gemv_mma(h, x, y, M, s);
         default:
             return set_error(BPDQ_ERR_INVALID, "bpdq_linear: unknown kernel id %d", kernel);
     }
@@ -215,6 +229,12 @@ extern "C" int bpdq_linear_batch(const bpdq_handle_t* hs, const void* const* xs,
     for (int k = 0; k < n; ++k)
         if (!xs[k] || !ys[k] || !aligned16(xs[k]) || !aligned16(ys[k]))
             return set_error(BPDQ_ERR_INVALID, "bpdq_linear_batch: x and y of linear %d must be non-null and 16-byte aligned", k);
+    // above the look-up-table threshold the few-token kernel takes the whole batch, when every linear allows it
+    bool few = M > hs[0]->gemv_max_m && M <= hs[0]->few_max_m && M <= BPDQ_FEW_MAX_M;
+    for (int k = 0; few && k < n; ++k)
+        few = hs[k]->d_few_maps && gemv_mma_supported(hs[k]->out, hs[k]->in, hs[k]->K, hs[k]->group) &&
+              (size_t)M * hs[k]->out * sizeof(float) <= hs[k]->ws_bytes;
+    if (few) return launch_gemv_mma_batch(hs, xs, ys, n, M, static_cast<cudaStream_t>(stream));
     return launch_gemv_batch(hs, xs, ys, n, M, static_cast<cudaStream_t>(stream));
 }
 
@@ -306,6 +326,14 @@ extern "C" int bpdq_set_gemv_max_m(bpdq_handle_t h, int max_gemv_m) {
     if (max_gemv_m < 0 || max_gemv_m > BPDQ_GEMV_MAX_M)
         return set_error(BPDQ_ERR_INVALID, "bpdq_set_gemv_max_m: %d outside [0, %d]", max_gemv_m, BPDQ_GEMV_MAX_M);
     h->gemv_max_m = max_gemv_m;
+    return BPDQ_OK;
+}
+
+extern "C" int bpdq_set_few_max_m(bpdq_handle_t h, int max_few_m) {
+    if (!h) return set_error(BPDQ_ERR_INVALID, "bpdq_set_few_max_m: null handle");
+    if (max_few_m < 0 || max_few_m > BPDQ_FEW_MAX_M)
+        return set_error(BPDQ_ERR_INVALID, "bpdq_set_few_max_m: %d outside [0, %d]", max_few_m, BPDQ_FEW_MAX_M);
+    h->few_max_m = max_few_m;
     return BPDQ_OK;
 }
 

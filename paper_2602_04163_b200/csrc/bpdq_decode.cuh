@@ -105,6 +105,16 @@ __device__ __forceinline__ void candidate_byte_tables(const float (&c)[K + 1], B
     }
 }
 
+// prmt.b32 as the hardware defines it: byte n of the result is byte (selector nibble n) & 7 of {b, a} (a = bytes 0..3);
+// a nibble with its top bit set would replicate that byte's sign instead.  Every selector used below keeps the top
+// bit of its four low nibbles clear (codes are at most 7), so no masking instruction is needed in front of it;
+// bits 16..31 of the selector are ignored.
+__device__ __forceinline__ unsigned prmt_raw(unsigned a, unsigned b, unsigned sel) {
+    unsigned d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
 // Four binary16 values from the four code nibbles in the low half of `sel`.
 template <int K>
 __device__ __forceinline__ void decode4(const unsigned sel, const ByteTables<K>& t, unsigned& out01, unsigned& out23) {
@@ -117,16 +127,16 @@ __device__ __forceinline__ void decode4(const unsigned sel, const ByteTables<K>&
         m = (m & 0x0011u) | ((m & 0x1100u) << 8);            // ... at 0, 4, 16, 20
         m = (m & 0x00010001u) | ((m & 0x00100010u) << 4);    // ... at 0, 8, 16, 24
         m *= 0xFFu;                                          // one full byte per code
-        const unsigned la = __byte_perm(t.lo[0], t.lo[1], s7), lb = __byte_perm(t.lo[2], t.lo[3], s7);
-        const unsigned ha = __byte_perm(t.hi[0], t.hi[1], s7), hb = __byte_perm(t.hi[2], t.hi[3], s7);
+        const unsigned la = prmt_raw(t.lo[0], t.lo[1], s7), lb = prmt_raw(t.lo[2], t.lo[3], s7);
+        const unsigned ha = prmt_raw(t.hi[0], t.hi[1], s7), hb = prmt_raw(t.hi[2], t.hi[3], s7);
         l = (la & ~m) | (lb & m);
         h = (ha & ~m) | (hb & m);
     } else {
-        l = __byte_perm(t.lo[0], t.lo[1], sel);
-        h = __byte_perm(t.hi[0], t.hi[1], sel);
+        l = prmt_raw(t.lo[0], t.lo[1], sel);
+        h = prmt_raw(t.hi[0], t.hi[1], sel);
     }
-    out01 = __byte_perm(l, h, 0x5140u);
-    out23 = __byte_perm(l, h, 0x7362u);
+    out01 = prmt_raw(l, h, 0x5140u);
+    out23 = prmt_raw(l, h, 0x7362u);
 }
 
 // Eight binary16 values (columns in order) from eight code nibbles.

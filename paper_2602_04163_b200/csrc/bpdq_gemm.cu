@@ -44,6 +44,7 @@
 // waits fall through, and the CTA still runs to its common exit where TMEM is freed.
 #include "bpdq_internal.h"
 #include "bpdq_decode.cuh"
+#include "bpdq_tma.cuh"
 
 #include <cuda.h>
 #include <cuda_fp16.h>
@@ -57,7 +58,6 @@ constexpr int kDecodeThreads = 128;               // per group: one thread per o
 constexpr int kThreads = 64 + kDecodeGroups * kDecodeThreads;
 constexpr int kTileThreads = 96 + kDecodeGroups * kDecodeThreads;   // tile kernel: producer warp, two MMA-issuing warps, eight decode warps
 constexpr int kATileBytes = BM * BK * 2;                       // 16 KB
-constexpr unsigned kWaitLimit = 1u << 24;                      // polls of try_wait before a wait gives up
 
 template <int K, int BN> struct Cfg {
     static constexpr int kBTileBytes = BN * BK * 2;
@@ -87,51 +87,11 @@ struct GemmParams {
     unsigned* counters;       // one arrival counter per 128-row tile, zero between calls
 };
 
-// ---- PTX wrappers ---------------------------------------------------------------------------
-__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false if the CTA has been aborted or the limit ran out (and aborts it).
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag, int* status) {
-    for (unsigned n = 0; n < kWaitLimit; ++n) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((n & 63u) == 63u && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    atomicExch(status, BPDQ_ERR_TIMEOUT);
-    return false;
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+// ---- PTX wrappers (mbarrier and TMA ones live in bpdq_tma.cuh) ------------------------------
+using namespace bpdq::tma;
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int c0, int c1, unsigned bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void bulk_load(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
 __device__ __forceinline__ void tmem_alloc(unsigned dst_smem, unsigned cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
 }
@@ -676,25 +636,8 @@ gemm_persistent_kernel(const __grid_constant__ CUtensorMap x_map, const GemmPara
 }
 
 // ---- host side ------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-        else
-            cudaGetLastError();
-    }
-    return fn;
-}
+using bpdq::EncodeTiledFn;
+using bpdq::encode_tiled_fn;
 
 template <int K, int BN>
 int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
@@ -799,6 +742,22 @@ int launch_k(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t strea
 }  // namespace
 
 namespace bpdq {
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
 
 bool gemm_supported(int, int, int K, int group) {
     return K >= 1 && K <= 4 && (group == 64 || group == 128 || group == 256);

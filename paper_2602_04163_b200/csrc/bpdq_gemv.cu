@@ -562,18 +562,19 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     int grid = h->sm_count < kMaxGrid ? h->sm_count : kMaxGrid;
     if ((long long)grid > total) grid = (int)total;
     const int kSegmentCost = p.n > 1 ? kSegmentCostBatch : kSegmentCostSingle;
-    static_assert(sizeof(h->plan_t_begin) == sizeof(p.t_begin), "one cached entry per CTA boundary");
-    bool cached = h->plan_n == p.n && h->plan_cost == kSegmentCost && h->plan_grid == grid;
-    for (int k = 0; cached && k < p.n; ++k) cached = h->plan_shape[k][0] == p.lin[k].nrg && h->plan_shape[k][1] == p.lin[k].nslices;
+    bpdq::LaunchPlan& plan = h->plan[0];
+    static_assert(sizeof(plan.t_begin) == sizeof(p.t_begin), "one cached entry per CTA boundary");
+    bool cached = plan.n == p.n && plan.cost == kSegmentCost && plan.grid == grid;
+    for (int k = 0; cached && k < p.n; ++k) cached = plan.shape[k][0] == p.lin[k].nrg && plan.shape[k][1] == p.lin[k].nslices;
     if (cached) {
-        for (int c = 0; c <= grid; ++c) p.t_begin[c] = h->plan_t_begin[c];
+        for (int c = 0; c <= grid; ++c) p.t_begin[c] = plan.t_begin[c];
     } else {
         int nrg[kMaxBatch], nsl[kMaxBatch];
         for (int k = 0; k < p.n; ++k) { nrg[k] = p.lin[k].nrg; nsl[k] = p.lin[k].nslices; }
         bpdq::cut_task_space(nrg, nsl, p.n, grid, kSegmentCost, p.t_begin);
-        h->plan_n = p.n; h->plan_cost = kSegmentCost; h->plan_grid = grid;
-        for (int k = 0; k < p.n; ++k) { h->plan_shape[k][0] = p.lin[k].nrg; h->plan_shape[k][1] = p.lin[k].nslices; }
-        for (int c = 0; c <= grid; ++c) h->plan_t_begin[c] = p.t_begin[c];
+        plan.n = p.n; plan.cost = kSegmentCost; plan.grid = grid;
+        for (int k = 0; k < p.n; ++k) { plan.shape[k][0] = p.lin[k].nrg; plan.shape[k][1] = p.lin[k].nslices; }
+        for (int c = 0; c <= grid; ++c) plan.t_begin[c] = p.t_begin[c];
     }
     p.dyn_smem = smem;
     cudaLaunchConfig_t cfg = {};

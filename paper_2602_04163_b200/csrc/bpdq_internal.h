@@ -52,6 +52,16 @@ inline int ensure_smem_optin(Kernel kernel, SmemOptin& rec, int device, int byte
 
 }  // namespace bpdq
 
+namespace bpdq {
+// Last cut of a launch's task space led by a handle (the cut depends on the shapes only): linears, their
+// (row groups, slices or column ranges), a key of the cost model, CTAs, first task of every CTA.  n == 0: none yet.
+struct LaunchPlan {
+    int n, cost, grid;
+    int shape[BPDQ_BATCH_MAX][2];
+    int t_begin[193];
+};
+}  // namespace bpdq
+
 struct bpdq_handle_s {
     int out, in, K, group, max_M, device;
     int sm_count;
@@ -68,14 +78,12 @@ struct bpdq_handle_s {
     void* d_ystage;
     int gemv_max_m;
     uint64_t launches;
-    // Last cut of a look-up-table launch led by this handle (the cut depends on the shapes only): linears,
-    // their (row groups, slices), segment cost, CTAs, first task of every CTA.  plan_n == 0: none yet.
+    int few_max_m;            // largest M the dispatcher sends to the few-token kernel
+    void* d_few_maps;         // device copy of the few-token kernel's two tensor maps (null: not available)
     // Tensor maps of the blob for the tensor-core kernel (planes, coefficients), encoded at the first launch.
     alignas(64) unsigned char gemm_maps[2][128];
     int gemm_maps_ready;
-    int plan_n, plan_cost, plan_grid;
-    int plan_shape[BPDQ_BATCH_MAX][2];
-    int plan_t_begin[193];
+    bpdq::LaunchPlan plan[2]; // [0] look-up-table kernel, [1] few-token kernel
 };
 
 // Kernel launchers (each returns a BPDQ_* status; all asynchronous on `stream`).
@@ -86,6 +94,10 @@ int launch_gemv_simple(bpdq_handle_s* h, const void* x, void* y, int M, cudaStre
 int launch_gemv(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
 int launch_gemv_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream);
 int launch_gemm(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
+int launch_gemv_mma(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
+int launch_gemv_mma_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream);
+bool gemv_mma_supported(int out, int in, int K, int group);
+int few_prepare(bpdq_handle_s* h);
 size_t gemv_workspace_bytes(int out, int in, int K, int group, int max_M, int sm_count);
 size_t gemv_counter_count(int out);
 bool gemv_supported(int out, int in, int K, int group);

@@ -19,7 +19,7 @@ def _run_batch(handles, xs_bits, M):
     return [y.cpu().numpy().astype(np.float64) for y in ys]
 
 
-@pytest.mark.parametrize("K,M", [(2, 1), (3, 2), (2, 5), (1, 1)])
+@pytest.mark.parametrize("K,M", [(2, 1), (3, 2), (2, 5), (1, 1), (3, 16), (4, 9)])
 def test_batch_matches_checker_and_single_launches(K, M):
     import oracle
     g = 128
@@ -33,7 +33,7 @@ def test_batch_matches_checker_and_single_launches(K, M):
         for (h, bits, coef), x, y in zip(layers, xs, ys):
             y_ref, a_ref = oracle.linear(bits, coef, x, g)
             G.assert_linear_close(y, y_ref, a_ref, f"batch rep {rep} {h.out}x{h.in_}")
-            y_single = G.run_linear(h, x, binding.KERNEL_GEMV)
+            y_single = G.run_linear(h, x, binding.KERNEL_AUTO)                # the same kernel as the batch takes for this M
             assert np.allclose(y, y_single, rtol=2.0 ** -9, atol=1e-5)
 
 
