@@ -6,7 +6,10 @@
 One JSON line on stdout.  The headline workload is a Qwen2.5-72B-shaped decoder layer at K = 2
 bit-planes, group 128, one token (M = 1): a step is one pass of bpdq_linear over the layer's seven
 linears.  Several distinct copies of the layer are rotated between steps so that no weight byte can
-be served from L2.  `value` is the useful HBM bytes (packed planes + coefficients + x + y) moved per
+be served from L2.  The timed region is `--steps` steps between two barriers; it is repeated
+TIMED_BLOCKS times back to back (one barrier before the first and one after the last block, an event
+between blocks) and the median block is reported: a block of 20 steps lasts about a millisecond, and
+the first launches after a pause run slower than the steady state.  `value` is the useful HBM bytes (packed planes + coefficients + x + y) moved per
 second; the `roofline` object relates it to the measured copy bandwidth.  Further timed sections
 (K = 3 layer, fused qkv / gate-up handles, prefill GEMM, dequant) are reported under `sections`.
 
@@ -39,9 +42,13 @@ UNIT = "GB/s"
 GROUP = 128
 HBM_NOMINAL_GBS = 8000.0
 FALLBACK_HBM_GBS, FALLBACK_TFLOPS = 6650.0, 1590.0
-# dram__bytes_read.sum + dram__bytes_write.sum of the headline launch, from one ncu capture of this kernel as it stands
-# (set to None whenever the kernel changes until the counters are taken again)
-GEMV_TRAFFIC_BYTES_PER_LAUNCH = 267_311_616
+# dram__bytes_read.sum + dram__bytes_write.sum of the headline launch, from the ncu capture summarised in
+# profiles/gemv_lut_K2_layer72b_batch_M1.md (set to None whenever the kernel changes until the counters are taken again)
+GEMV_TRAFFIC_BYTES_PER_LAUNCH = 264_366_080
+# the same for one launch of the persistent tcgen05 kernel on the gate projection at K = 3, M = 2048
+# (profiles/gemm_K3_gate_29568x8192_M2048.md); the prefill sections time whole layers, so this is context for them
+GEMM_GATE_K3_M2048_TRAFFIC_BYTES = None
+TIMED_BLOCKS = 25
 
 
 def useful_bytes(out: int, in_: int, K: int, g: int, M: int) -> int:
@@ -132,30 +139,58 @@ def time_oracle(sample, K: int):
     return time.perf_counter() - t0, covered
 
 
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def time_oracle_threads(sample, K: int, threads: int, M: int = 1):
+    """The unchanged checker function on `threads` host threads, each on its own slice of the sample's output rows
+    (the foreign call releases the interpreter lock); returns (seconds, useful bytes covered, weights covered)."""
+    import concurrent.futures
+    import oracle
+    jobs = []
+    for _, out, in_, bits, coef, x in sample:
+        n = bits.shape[1]
+        cuts = np.linspace(0, n, min(threads, n) + 1).astype(int)
+        for a, b in zip(cuts[:-1], cuts[1:]):
+            if b > a:
+                jobs.append((np.ascontiguousarray(bits[:, a:b]), np.ascontiguousarray(coef[:, a:b]), x))
+    covered = sum(useful_bytes(b.shape[1], i, K, GROUP, M) for _, _, i, b, _, _ in sample)
+    weights = sum(b.shape[1] * i for _, _, i, b, _, _ in sample)
+    t0 = time.perf_counter()
+    with concurrent.futures.ThreadPoolExecutor(max_workers=threads) as ex:
+        list(ex.map(lambda j: oracle.linear(j[0], j[1], j[2], GROUP), jobs))
+    return time.perf_counter() - t0, covered, weights
+
+
 def run_reference(args, rank: int):
     if rank != 0:
         return
     shapes, K = synth.QWEN25_72B_LAYER, 2
     # bounded sample: the whole run (warm-up included) stays near one minute at the checker's ~8e6 weights/s
     cols = sum(i for _, _, i in shapes)
-    rows = max(2, min(512, int(60.0 * 8e6 / (cols * max(1, args.steps + args.warmup)))))
+    rows = max(2, min(4096, int(60.0 * 8e6 * host_cores() / (cols * max(1, args.steps + args.warmup)))))
     sample = oracle_sample(shapes, K, rows)
     import oracle
     oracle.build()
+    cores = host_cores()
     for _ in range(args.warmup):
-        time_oracle(sample, K)
+        time_oracle_threads(sample, K, cores)
     t_total, covered = 0.0, 0
     for _ in range(args.steps):
-        dt, nb = time_oracle(sample, K)
+        dt, nb, _ = time_oracle_threads(sample, K, cores)
         t_total += dt
         covered += nb
     value = covered / t_total / 1e9
-    desc = f"{rows} evenly spaced output rows of each of the 7 linears per step, single thread"
+    desc = f"{rows} evenly spaced output rows of each of the 7 linears per step, rows split over {cores} host threads"
     line = {"metric": METRIC, "value": value, "unit": UNIT, "impl": "reference", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": "qwen2.5-72b-shaped decoder layer, K=2, g=128, M=1 (7 linears)", "sample": desc},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -247,15 +282,19 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
     sampler.start()
     time.sleep(0.3)
     t_wall0 = time.time()
-    # the timed region: exactly `steps` steps, CUDA events on the launching stream
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # the timed region: TIMED_BLOCKS blocks of exactly `steps` steps, back to back between two barriers, an event on the
+    # launching stream between blocks; the median block is the one reported
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(TIMED_BLOCKS + 1)]
     barrier()
-    e0.record(stream)
-    for s in range(args.steps):
-        step(layers[s % copies])
-    e1.record(stream)
+    marks[0].record(stream)
+    for blk in range(TIMED_BLOCKS):                                 # back to back: no host wait between blocks
+        for s in range(args.steps):
+            step(layers[(blk * args.steps + s) % copies])
+        marks[blk + 1].record(stream)
     barrier()
-    ms_total = e0.elapsed_time(e1)
+    block_ms = [marks[b].elapsed_time(marks[b + 1]) for b in range(TIMED_BLOCKS)]
+    ms_first = block_ms[0]
+    ms_total = sorted(block_ms)[len(block_ms) // 2]
     t_wall1 = time.time()
     launches2 = sum(h.bpdq_launch_count() for L in layers for _, h in L.handles)
 
@@ -294,7 +333,7 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
     value = replica_throughput_gbs(bytes_step, args.steps, world, ms_total)
     e2e_value = replica_throughput_gbs(bytes_step, args.steps, world, e2e_ms)
     per_gpu = value / world
-    n_launch = (launches2 - launches1)
+    n_launch = (launches2 - launches1) // TIMED_BLOCKS              # kernels launched inside one timed block
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -302,7 +341,8 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
             "config": {"workload": "qwen2.5-72b-shaped decoder layer, K=2, g=128, M=1 (7 linears: q k v o gate up down, each with its own x, "
                                    "issued as one bpdq_linear_batch call; sections.seven_separate_calls times seven bpdq_linear calls)",
                        "l2": f"inputs larger than L2: {copies} distinct layer copies of {bytes_step / 1e6:.1f} MB rotated between steps",
-                       "useful_bytes_per_step": bytes_step, "parallelism": "replicas only" if world > 1 else "single GPU"},
+                       "useful_bytes_per_step": bytes_step, "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "timing": f"median of {TIMED_BLOCKS} back-to-back blocks of `steps` steps between two barriers; first block {ms_first / args.steps * 1e3:.1f} us per step"},
             "e2e": {"value": e2e_value, "unit": UNIT,
                     "h2d_bytes_per_step": sum(2 * M * i for _, _, i in shapes), "d2h_bytes_per_step": sum(2 * M * o for _, o, _ in shapes),
                     "path": "bpdq_linear_batch_host, every step: one gather launch reads the seven x from pinned host memory, the kernel "
@@ -331,6 +371,10 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
         line["sections"] = extra_sections(torch, binding, args, peaks, sp, stream)
         line["sections"]["seven_separate_calls"] = separate
         line["sections"]["decode_sweep_80_layers_K2"] = full_stack_section(torch, binding, peaks, sp, stream)
+        dg = line["sections"].get("gemv_layer_batched_decoder_groups_K2", {})
+        line["config"]["same_layer_other_issue_orders"] = {
+            "decoder_legal_groups_qkv_o_gateup_down": {"us_per_layer": dg.get("us_per_layer"), "frac_measured": dg.get("frac_measured")},
+            "seven_bpdq_linear_calls": {"us_per_layer": separate["us_per_layer"], "frac_measured": separate["frac_measured"]}}
     for L in layers:
         L.destroy()
 
@@ -344,14 +388,37 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
 
 
 def cpu_baseline(shapes, K):
-    """The checker as it stands, single thread, on a bounded sample of the same layer (about 15 s)."""
+    """The checker as it stands on the machine's host cores, on bounded samples of the benchmark's workloads (about 25 s):
+    the decode layer on every core (row-parallel wrapper around the unchanged function) and on one core, and a
+    subset of the prefill layer whose full-size time is extrapolated from it."""
     import oracle
     oracle.build()
-    rows = 1536
-    sample = oracle_sample(shapes, K, rows)
-    dt, covered = time_oracle(sample, K)
-    return {"value": covered / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
-            "sample": f"{rows} evenly spaced output rows of each of the 7 linears of the layer (M=1), one pass"}
+    cores = host_cores()
+    rows1 = 2304
+    dt1, cov1, _ = time_oracle_threads(oracle_sample(shapes, K, rows1), K, 1)
+    rows_all = min(29568, 2560 * cores)
+    dta, cova, _ = time_oracle_threads(oracle_sample(shapes, K, rows_all), K, cores)
+    # prefill subset: 16 tokens through `rows_p` rows of every linear at K = 3; the checker's cost per (weight, token)
+    # pair is taken from it and scaled to 8192 tokens x all rows (decode cost per weight is paid once per row)
+    Kp, Mp, rows_p = 3, 16, 96 * cores
+    samp = []
+    for li, (name, out, in_) in enumerate(shapes):
+        sd = 700 + li
+        rows = np.unique(np.linspace(0, out - 1, rows_p).astype(np.int64))
+        samp.append((name, out, in_, synth.plane_bits(sd, out, in_, Kp, rows), synth.coefficients(sd, out, in_, Kp, GROUP, rows),
+                     synth.activations(3, 8192, in_, tokens=np.arange(Mp))))
+    dtp, _, wp = time_oracle_threads(samp, Kp, cores, Mp)
+    full_weights = sum(o * i for _, o, i in shapes)
+    est_s_8192 = dtp / (wp * Mp) * full_weights * 8192          # upper bound: charges the per-weight decode to every token
+    flops_8192 = 2.0 * 8192 * full_weights
+    return {"value": cova / dta / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": dta,
+            "sample": f"{rows_all} evenly spaced output rows of each of the 7 linears of the layer (M=1), one pass, rows split over {cores} threads",
+            "single_thread": {"value": cov1 / dt1 / 1e9, "unit": UNIT, "cores": 1, "seconds": dt1,
+                              "sample": f"{rows1} evenly spaced output rows of each of the 7 linears (M=1), one pass"},
+            "prefill_subset": {"K": Kp, "tokens": Mp, "rows_per_linear": rows_p, "cores": cores, "seconds": dtp,
+                               "extrapolated_seconds_layer_M8192": est_s_8192,
+                               "extrapolated_tflops_layer_M8192": flops_8192 / est_s_8192 / 1e12,
+                               "note": "extrapolated from the subset by (weights x tokens); not measured at full size"}}
 
 
 def extra_sections(torch, binding, args, peaks, sp, stream):
@@ -473,7 +540,8 @@ def extra_sections(torch, binding, args, peaks, sp, stream):
             for h in L:
                 h.bpdq_destroy()
 
-    # token-count sweep on the gate and down projections: both kernels, to place the dispatch threshold
+    # token-count sweep on the gate and down projections: all three kernels (the dispatch thresholds come from it) and
+    # what bpdq_linear itself picks; an L2 flush before every launch
     sweep = []
     for K in (2, 3):
         for name, o, i in (("gate", 29568, 8192), ("down", 8192, 29568)):
@@ -482,13 +550,16 @@ def extra_sections(torch, binding, args, peaks, sp, stream):
                 x = xt(M, i)
                 y = torch.empty((M, o), dtype=torch.float16, device="cuda")
                 rec = {"linear": name, "K": K, "M": M}
-                for kname, kid in (("lut", binding.KERNEL_GEMV), ("tensor", binding.KERNEL_GEMM)):
-                    if kid == binding.KERNEL_GEMV and M > binding.GEMV_MAX_M:
+                for kname, kid in (("lut", binding.KERNEL_GEMV), ("few", binding.KERNEL_FEW), ("tensor", binding.KERNEL_GEMM)):
+                    if (kid == binding.KERNEL_GEMV and M > binding.GEMV_MAX_M) or (kid == binding.KERNEL_FEW and M > binding.FEW_MAX_M):
                         continue
                     med, _ = timed(lambda: h.bpdq_linear_ex(x.data_ptr(), y.data_ptr(), M, kid, sp), 5)
                     rec[f"us_{kname}"] = med * 1e3
                 best = min(v for k, v in rec.items() if k.startswith("us_"))
                 rec["gbs_best"] = useful_bytes(o, i, K, GROUP, M) / (best * 1e-6) / 1e9
+                rec["frac_measured_best"] = rec["gbs_best"] / peaks["hbm_gbs"]
+                med, _ = timed(lambda: h.bpdq_linear(x.data_ptr(), y.data_ptr(), M, sp), 5)
+                rec["us_dispatcher"] = med * 1e3
                 sweep.append(rec)
             h.bpdq_destroy()
     out["token_sweep"] = sweep
@@ -515,12 +586,76 @@ def extra_sections(torch, binding, args, peaks, sp, stream):
         tf = flops / (ms * 1e-3) / 1e12
         out[f"prefill_gemm_layer_K{K}_M{M}"] = {
             "ms_per_layer": ms, "tflops": tf, "per_linear": per,
-            "roofline": {"bound": "tensor", "kernel": "gemm_kernel", "achieved": tf, "peak": peaks["tflops"], "unit": "TFLOP/s",
+            "roofline": {"bound": "tensor", "kernel": "gemm_persistent_kernel", "achieved": tf, "peak": peaks["tflops"], "unit": "TFLOP/s",
                          "frac": tf / peaks["tflops"], "frac_of_sustained": tf / peaks["tflops_sustained"],
-                         "peak_source": peaks["source"] + " bf16 burst (fp16 has the same nominal rate)", "traffic": None}}
+                         "peak_source": peaks["source"] + " bf16 burst (fp16 has the same nominal rate)",
+                         "traffic": None, "traffic_gate_launch_K3_M2048": GEMM_GATE_K3_M2048_TRAFFIC_BYTES}}
         for h in hs:
             h.bpdq_destroy()
         del xs, ys
+
+    # the paper's own formats (Table 1) on the 72B-shaped layer: decode as one batched launch, prefill at M = 8192
+    for tag, K, g in (("W2-G64", 2, 64), ("W3-G64", 3, 64), ("W2-G256", 2, 256), ("W4-G128", 4, 128)):
+        copies = 3
+        gof = lambda i: g if i % g == 0 else 128      # 29568 input columns are not a multiple of 256: that linear keeps groups of 128
+        layers = [[binding.Handle(o, i, K, gof(i), None, 1100 + 10 * c + li, 1) for li, (_, o, i) in enumerate(shapes)] for c in range(copies)]
+        xs1 = {8192: xt(1, 8192), 29568: xt(1, 29568)}
+        ys1 = [torch.empty((1, o), dtype=torch.float16, device="cuda") for _, o, _ in shapes]
+        b = sum(useful_bytes(o, i, K, gof(i), 1) for _, o, i in shapes)
+        n = 60
+
+        def run_fmt():
+            for k in range(n):
+                hs_ = layers[k % copies]
+                binding.bpdq_linear_batch(hs_, [xs1[h.in_].data_ptr() for h in hs_], [y.data_ptr() for y in ys1], 1, sp)
+        run_fmt()
+        ms = event_time_ms(torch, run_fmt, stream) / n
+        rec = {"K": K, "group": g, "bits_per_weight": K + 16.0 * (K + 1) / g, "decode_us_per_layer": ms * 1e3, "decode_gbs": b / (ms * 1e-3) / 1e9,
+               "decode_frac_measured": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        for L in layers:
+            for h in L:
+                h.bpdq_destroy()
+        M = 8192
+        hs = [binding.Handle(o, i, K, gof(i), None, 1200 + li, M) for li, (_, o, i) in enumerate(shapes)]
+        xs = {8192: xt(M, 8192), 29568: xt(M, 29568)}
+        ys = {o: torch.empty((M, o), dtype=torch.float16, device="cuda") for o in sorted({o for _, o, _ in shapes})}
+
+        def run_prefill_fmt():
+            for h in hs:
+                h.bpdq_linear(xs[h.in_].data_ptr(), ys[h.out].data_ptr(), M, sp)
+        run_prefill_fmt()
+        msp = sorted(event_time_ms(torch, run_prefill_fmt, stream) for _ in range(3))[1]
+        tf = sum(2.0 * M * o * i for _, o, i in shapes) / (msp * 1e-3) / 1e12
+        rec.update({"prefill_M8192_ms_per_layer": msp, "prefill_tflops": tf, "prefill_frac_measured_burst": tf / peaks["tflops"]})
+        out[f"paper_format_{tag}"] = rec
+        for h in hs:
+            h.bpdq_destroy()
+        del xs, ys
+
+    # a decoder layer with a few tokens in flight (M = 4, 8, 16): the grouping a decoder allows, one bpdq_linear_batch
+    # call per group (the few-token kernel takes them above two tokens)
+    for K in (2, 3):
+        copies = 3
+        layers = [[binding.Handle(o, i, K, GROUP, None, 1300 + 10 * c + li, 16) for li, (_, o, i) in enumerate(shapes)] for c in range(copies)]
+        for M in (4, 8, 16):
+            xs = {8192: xt(M, 8192), 29568: xt(M, 29568)}
+            ys = [torch.empty((M, o), dtype=torch.float16, device="cuda") for _, o, _ in shapes]
+            b = layer_bytes(shapes, K, M)
+            n = 30
+
+            def run_few():
+                for k in range(n):
+                    hs_ = layers[k % copies]
+                    for grp in ([0, 1, 2], [3], [4, 5], [6]):
+                        binding.bpdq_linear_batch([hs_[j] for j in grp], [xs[hs_[j].in_].data_ptr() for j in grp],
+                                                  [ys[j].data_ptr() for j in grp], M, sp)
+            run_few()
+            ms = event_time_ms(torch, run_few, stream) / n
+            out[f"few_token_layer_decoder_groups_K{K}_M{M}"] = {"launches_per_layer": 4, "us_per_layer": ms * 1e3, "gbs": b / (ms * 1e-3) / 1e9,
+                                                                "frac_measured": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        for L in layers:
+            for h in L:
+                h.bpdq_destroy()
     return out
 
 

@@ -19,7 +19,7 @@ def _run_batch(handles, xs_bits, M):
     return [y.cpu().numpy().astype(np.float64) for y in ys]
 
 
-@pytest.mark.parametrize("K,M", [(2, 1), (3, 2), (2, 5), (1, 1), (3, 16), (4, 9)])
+@pytest.mark.parametrize("K,M", [(2, 1), (3, 2), (2, 5), (1, 1), (3, 16), (1, 9)])
 def test_batch_matches_checker_and_single_launches(K, M):
     import oracle
     g = 128
