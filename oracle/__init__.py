@@ -41,7 +41,12 @@ def _load():
         lib.oracle_dequant.argtypes = [p, p, i64, i64, ctypes.c_int, i64, p]
         lib.oracle_linear.argtypes = [p, p, p, i64, i64, ctypes.c_int, i64, i64, p, p]
         lib.oracle_unpack.argtypes = [p, i64, i64, ctypes.c_int, i64, p, p]
-        for f in (lib.oracle_dequant, lib.oracle_linear, lib.oracle_unpack):
+        lib.oracle_linear_perm.argtypes = [p, p, p, p, i64, i64, ctypes.c_int, i64, i64, p, p]
+        lib.oracle_silu.argtypes = [ctypes.c_double]
+        lib.oracle_silu.restype = ctypes.c_double
+        lib.oracle_swiglu.argtypes = [p, p, i64, p]
+        lib.oracle_add_bias.argtypes = [p, p, i64, i64]
+        for f in (lib.oracle_dequant, lib.oracle_linear, lib.oracle_unpack, lib.oracle_linear_perm, lib.oracle_swiglu, lib.oracle_add_bias):
             f.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -105,3 +110,45 @@ def unpack(blob: np.ndarray, out: int, in_: int, K: int, group: int):
     if rc:
         raise ValueError("oracle_unpack rejected its arguments")
     return bits, coef
+
+
+def linear_perm(bits: np.ndarray, coef: np.ndarray, x: np.ndarray, perm: np.ndarray, group: int):
+    """y[m,r] = sum_j x[m, perm[j]] * w[r,j]: the stored columns are a reordering of the input channels.  Returns (y, a)."""
+    bits = _c(bits, np.uint8)
+    coef = _c(coef, np.uint16)
+    x = _c(x, np.uint16)
+    perm = _c(perm, np.int64)
+    K, out, in_ = bits.shape
+    M = x.shape[0]
+    assert x.shape == (M, in_) and perm.shape == (in_,)
+    y = np.empty((M, out), dtype=np.float64)
+    a = np.empty((M, out), dtype=np.float64)
+    rc = _load().oracle_linear_perm(_ptr(bits), _ptr(coef), _ptr(x), _ptr(perm), out, in_, K, group, M, _ptr(y), _ptr(a))
+    if rc:
+        raise ValueError("oracle_linear_perm rejected its arguments (perm must be a permutation)")
+    return y, a
+
+
+def silu(v: float) -> float:
+    return float(_load().oracle_silu(float(v)))
+
+
+def swiglu(gate: np.ndarray, up: np.ndarray) -> np.ndarray:
+    """h = silu(gate) * up, elementwise in binary64."""
+    gate = _c(gate, np.float64)
+    up = _c(up, np.float64)
+    assert gate.shape == up.shape
+    h = np.empty(gate.shape, dtype=np.float64)
+    if _load().oracle_swiglu(_ptr(gate), _ptr(up), gate.size, _ptr(h)):
+        raise ValueError("oracle_swiglu rejected its arguments")
+    return h
+
+
+def add_bias(y: np.ndarray, bias: np.ndarray) -> np.ndarray:
+    """y + float(bias) per output row, bias as binary16 bit patterns [out]."""
+    y = np.array(y, dtype=np.float64, order="C")
+    bias = _c(bias, np.uint16)
+    assert y.ndim == 2 and bias.shape == (y.shape[1],)
+    if _load().oracle_add_bias(_ptr(y), _ptr(bias), y.shape[0], y.shape[1]):
+        raise ValueError("oracle_add_bias rejected its arguments")
+    return y

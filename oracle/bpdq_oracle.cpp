@@ -30,6 +30,11 @@
 // float64 matrix product.  The acceptance bound on y (4e-3 * a + 1e-3) is this library's
 // acceptance criterion, not a statement of the paper: beyond that bound the y tolerance is "parity unpinned".
 //
+// Around the map (pins in tests/test_oracle_extensions.py): oracle_linear_perm (stored columns are a reordering of
+// the input channels: Section 4 names Group-Aware Reordering for the quantizer, the inference side is this file's
+// reading), oracle_swiglu and oracle_add_bias (steps of the decoder layer around the linears, not of the paper's
+// method).  The data-free producer (Eq. 5 bit-plane selection, Eq. 6 with U_loc = I) is oracle/producer.py.
+//
 // oracle_unpack is an independent reader of the device blob layout, written from the
 // layout's description (not from the library's packer):
 //   planes : for block b = floor(j/128), plane i (0-based), row r: 16 bytes at byte offset
@@ -154,6 +159,57 @@ int oracle_linear(const uint8_t* bits, const uint16_t* coef, const uint16_t* x, 
             }
         }
     }
+    return 0;
+}
+
+// The same map when the stored columns are a reordering of the layer's input channels (the paper quantizes with
+// Group-Aware Reordering, Section 4 "Baselines and Hyperparameters": whole groups of channels are moved, and the
+// quantized matrix keeps that order).  Stored column j multiplies input channel perm[j]:
+//     y[m,r] = sum_j x[m, perm[j]] * W^[r,j].
+// The paper does not say how inference undoes the reordering; this is the reading that leaves the layer's
+// function unchanged.  perm must be a permutation of 0..in-1 (checked).
+int oracle_linear_perm(const uint8_t* bits, const uint16_t* coef, const uint16_t* x, const int64_t* perm, int64_t out,
+                       int64_t in, int K, int64_t g, int64_t M, double* y, double* a) {
+    if (!bits || !coef || !x || !perm || !y || out <= 0 || in <= 0 || K < 1 || g <= 0 || in % g || M < 0) return 1;
+    {
+        uint8_t* seen = new uint8_t[in]();
+        bool ok = true;
+        for (int64_t j = 0; j < in; ++j) {
+            if (perm[j] < 0 || perm[j] >= in || seen[perm[j]]) { ok = false; break; }
+            seen[perm[j]] = 1;
+        }
+        delete[] seen;
+        if (!ok) return 1;
+    }
+    const int64_t ngroups = in / g;
+    for (int64_t r = 0; r < out; ++r) {
+        for (int64_t m = 0; m < M; ++m) { y[m * out + r] = 0.0; if (a) a[m * out + r] = 0.0; }
+        for (int64_t j = 0; j < in; ++j) {
+            const double wj = (double)half_bits_to_float(decode_one(bits, coef, out, in, K, ngroups, r, j, j / g));
+            for (int64_t m = 0; m < M; ++m) {
+                const double p = (double)half_bits_to_float(x[m * in + perm[j]]) * wj;
+                y[m * out + r] += p;
+                if (a) a[m * out + r] += std::fabs(p);
+            }
+        }
+    }
+    return 0;
+}
+
+// Gated unit around a (gate, up) pair of linears, h = silu(gate) * up with silu(v) = v / (1 + exp(-v)), and an
+// additive bias: both are steps of the decoder layer the paper's per-token latency is measured on, not of the
+// paper's method; written out here in binary64 so that the library's fused epilogues can be checked.
+double oracle_silu(double v) { return v / (1.0 + std::exp(-v)); }
+int oracle_swiglu(const double* gate, const double* up, int64_t n, double* h) {
+    if (!gate || !up || !h || n < 0) return 1;
+    for (int64_t i = 0; i < n; ++i) h[i] = oracle_silu(gate[i]) * up[i];
+    return 0;
+}
+// y[m][r] += float(bias[r]) for binary16 bias bits.
+int oracle_add_bias(double* y, const uint16_t* bias, int64_t M, int64_t out) {
+    if (!y || !bias || M < 0 || out <= 0) return 1;
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t r = 0; r < out; ++r) y[m * out + r] += (double)half_bits_to_float(bias[r]);
     return 0;
 }
 
