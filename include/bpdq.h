@@ -113,6 +113,25 @@ BPDQ_API int bpdq_pack(const uint8_t* bits, const uint16_t* coef, int out, int i
 BPDQ_API int bpdq_unpack(const void* blob, int out, int in, int K, int group, uint8_t* bits,
                 uint16_t* coef);
 
+/* Data-free producer of logical tensors from full-precision weights w (host, binary32 [out][in]): the
+ * initialisation of the paper's quantizer without calibration data.  Per (row, group): asymmetric
+ * round-to-nearest (ties to even) to an unsigned 8-bit code with scale (max - min) / 255 (paper:
+ * Section 3.2, Eq. 5, Z = sum 2^i P_i); bits[i-1] = B_i = P_{7-K+i}, the K most significant planes;
+ * coefficients by Eq. 6 with U_loc = I (least squares of the weights on [1, b_1, .., b_K], normal
+ * equations in binary64, alpha * trace / (K+1) added to the diagonal; the paper uses alpha = 1e-4),
+ * rounded to binary16.  bits / coef as for bpdq_pack.  Host only, no CUDA call.  NaN weights are
+ * BPDQ_ERR_INVALID. */
+BPDQ_API int bpdq_quantize_datafree(const float* w, int out, int in, int K, int group, double alpha, uint8_t* bits,
+                           uint16_t* coef);
+
+/* Multi-precision view (paper: closing section, serving several precisions from one stored model;
+ * the mechanism is this library's reading): from logical tensors with K planes, those with the K2
+ * most significant planes B_{K-K2+1}..B_K and their coefficients; every dropped plane adds half its
+ * coefficient to the offset (binary32 adds in plane order, one rounding to binary16).  bits2
+ * [K2][out][in], coef2 [K2+1][out][in/g] are caller-owned and may alias nothing.  Host only. */
+BPDQ_API int bpdq_truncate_planes(const uint8_t* bits, const uint16_t* coef, int out, int in, int K, int group, int K2,
+                         uint8_t* bits2, uint16_t* coef2);
+
 /* Creates a layer on the current CUDA device.  `host_blob` (host memory, bpdq_packed_bytes()
  * bytes) is copied to the device; if it is NULL the blob is generated on the device from
  * `seed` with the counter-based generator of the synthetic workloads (plane bits iid

@@ -23,7 +23,7 @@ NOALLOC_MAX_OUT = 65536
 
 EXPORTS = ("bpdq_packed_bytes", "bpdq_pack", "bpdq_unpack", "bpdq_create", "bpdq_dequant", "bpdq_linear",
            "bpdq_linear_ex", "bpdq_linear_host", "bpdq_set_gemv_max_m", "bpdq_set_few_max_m", "bpdq_read_blob", "bpdq_get_status",
-           "bpdq_launch_count", "bpdq_destroy", "bpdq_last_error", "bpdq_linear_noalloc", "bpdq_linear_batch", "bpdq_linear_batch_host")
+           "bpdq_launch_count", "bpdq_destroy", "bpdq_quantize_datafree", "bpdq_truncate_planes", "bpdq_last_error", "bpdq_linear_noalloc", "bpdq_linear_batch", "bpdq_linear_batch_host")
 
 _lib = None
 
@@ -47,6 +47,8 @@ def lib() -> ctypes.CDLL:
         L.bpdq_packed_bytes.restype = ctypes.c_size_t
         L.bpdq_pack.argtypes = [vp, vp, i, i, i, i, vp]
         L.bpdq_unpack.argtypes = [vp, i, i, i, i, vp, vp]
+        L.bpdq_quantize_datafree.argtypes = [vp, i, i, i, i, ctypes.c_double, vp, vp]
+        L.bpdq_truncate_planes.argtypes = [vp, vp, i, i, i, i, i, vp, vp]
         L.bpdq_create.argtypes = [ctypes.POINTER(vp), i, i, i, i, vp, u64, i]
         L.bpdq_dequant.argtypes = [vp, vp, vp]
         L.bpdq_linear.argtypes = [vp, vp, vp, i, vp]
@@ -110,6 +112,27 @@ def bpdq_unpack(blob: np.ndarray, out: int, in_: int, K: int, group: int):
     coef = np.empty((K + 1, out, in_ // group), dtype=np.uint16)
     _check(lib().bpdq_unpack(_np_ptr(blob), out, in_, K, group, _np_ptr(bits), _np_ptr(coef)))
     return bits, coef
+
+
+def bpdq_quantize_datafree(w: np.ndarray, K: int, group: int, alpha: float = 1e-4):
+    """w float32 [out][in] -> (bits uint8 [K][out][in], coef uint16 [K+1][out][in/group])."""
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    out, in_ = w.shape
+    bits = np.empty((K, out, in_), dtype=np.uint8)
+    coef = np.empty((K + 1, out, in_ // group), dtype=np.uint16)
+    _check(lib().bpdq_quantize_datafree(_np_ptr(w), out, in_, K, group, alpha, _np_ptr(bits), _np_ptr(coef)))
+    return bits, coef
+
+
+def bpdq_truncate_planes(bits: np.ndarray, coef: np.ndarray, group: int, K2: int):
+    """The view with the K2 most significant planes of (bits, coef)."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint8)
+    coef = np.ascontiguousarray(coef, dtype=np.uint16)
+    K, out, in_ = bits.shape
+    bits2 = np.empty((K2, out, in_), dtype=np.uint8)
+    coef2 = np.empty((K2 + 1, out, in_ // group), dtype=np.uint16)
+    _check(lib().bpdq_truncate_planes(_np_ptr(bits), _np_ptr(coef), out, in_, K, group, K2, _np_ptr(bits2), _np_ptr(coef2)))
+    return bits2, coef2
 
 
 def bpdq_linear_noalloc(blob_ptr: int, out: int, in_: int, K: int, group: int, x_ptr: int, y_ptr: int, M: int,
