@@ -215,6 +215,33 @@ BPDQ_API int bpdq_linear_host(bpdq_handle_t h, const void* x_fp16_host, void* y_
 BPDQ_API int bpdq_linear_noalloc(const void* blob_dev, int out, int in, int K, int group, const void* x_fp16_dev,
                         void* y_fp16_dev, int M, void* stream);
 
+/* Input-channel permutation (paper: Section 4, the quantizer reorders channels with Group-Aware
+ * Reordering and keeps the quantized matrix in that order; how inference undoes it is this
+ * library's reading).  With perm set (host, int32 [in], a permutation of 0..in-1; copied), every
+ * linear call on the handle computes y[m,r] = sum_j x[m, perm[j]] * W^[r,j]: the look-up-table
+ * kernel reads x through perm while it builds its tables, the other kernels run on a gathered copy
+ * of x that one extra launch writes into a handle-owned buffer.  NULL restores the identity.
+ * Synchronises the device. */
+BPDQ_API int bpdq_set_input_permutation(bpdq_handle_t h, const int32_t* perm_host);
+
+/* Bias (not part of the paper's method; decoder layers carry one on q, k and v): binary16 [out] on
+ * the host, copied; added in binary32 to every output row before the rounding to binary16, in
+ * every kernel.  NULL removes it.  Synchronises the device. */
+BPDQ_API int bpdq_set_bias(bpdq_handle_t h, const uint16_t* bias_fp16_host);
+
+/* The gated unit around a (gate, up) pair that shares its input: h[m,r] = silu(g) * u with
+ * g = x W^gate^T (+ bias), u = x W^up^T (+ bias), silu(v) = v / (1 + exp(-v)), evaluated in binary32
+ * and rounded to binary16 (not part of the paper's method: the step that follows these two
+ * linears in the decoder layers the paper measures).  Both handles have
+ * the same out, in and K and live on the current device; 0 <= M <= min(max_M).  Up to the
+ * few-token threshold the two linears run in one launch and the kernel that completes a block of
+ * rows applies the unit to the unrounded binary32 sums (nothing but h is written); above it two
+ * tcgen05 launches write g and u, rounded to binary16, to handle-owned buffers and a third launch
+ * applies the unit.  x, h_out: device binary16 [M][in] /
+ * [M][out], 16-byte aligned. */
+BPDQ_API int bpdq_gate_up_swiglu(bpdq_handle_t gate, bpdq_handle_t up, const void* x_fp16_dev, void* h_fp16_dev, int M,
+                        void* stream);
+
 /* Sets the largest M that bpdq_linear sends to the look-up-table kernel (0 = always use the
  * tensor-core kernel; at most BPDQ_GEMV_MAX_M). */
 BPDQ_API int bpdq_set_gemv_max_m(bpdq_handle_t h, int max_gemv_m);

@@ -23,7 +23,7 @@ NOALLOC_MAX_OUT = 65536
 
 EXPORTS = ("bpdq_packed_bytes", "bpdq_pack", "bpdq_unpack", "bpdq_create", "bpdq_dequant", "bpdq_linear",
            "bpdq_linear_ex", "bpdq_linear_host", "bpdq_set_gemv_max_m", "bpdq_set_few_max_m", "bpdq_read_blob", "bpdq_get_status",
-           "bpdq_launch_count", "bpdq_destroy", "bpdq_quantize_datafree", "bpdq_truncate_planes", "bpdq_last_error", "bpdq_linear_noalloc", "bpdq_linear_batch", "bpdq_linear_batch_host")
+           "bpdq_launch_count", "bpdq_destroy", "bpdq_quantize_datafree", "bpdq_truncate_planes", "bpdq_set_input_permutation", "bpdq_set_bias", "bpdq_gate_up_swiglu", "bpdq_last_error", "bpdq_linear_noalloc", "bpdq_linear_batch", "bpdq_linear_batch_host")
 
 _lib = None
 
@@ -59,6 +59,9 @@ def lib() -> ctypes.CDLL:
         L.bpdq_linear_noalloc.argtypes = [vp, i, i, i, i, vp, vp, i, vp]
         L.bpdq_set_gemv_max_m.argtypes = [vp, i]
         L.bpdq_set_few_max_m.argtypes = [vp, i]
+        L.bpdq_set_input_permutation.argtypes = [vp, vp]
+        L.bpdq_set_bias.argtypes = [vp, vp]
+        L.bpdq_gate_up_swiglu.argtypes = [vp, vp, vp, vp, i, vp]
         L.bpdq_read_blob.argtypes = [vp, vp]
         L.bpdq_get_status.argtypes = [vp, vp]
         L.bpdq_launch_count.argtypes = [vp, ctypes.POINTER(u64)]
@@ -135,6 +138,11 @@ def bpdq_truncate_planes(bits: np.ndarray, coef: np.ndarray, group: int, K2: int
     return bits2, coef2
 
 
+def bpdq_gate_up_swiglu(gate, up, x_ptr: int, h_ptr: int, M: int, stream: int = 0) -> None:
+    """h = silu(x Wgate^T) * (x Wup^T) for two handles that share their input."""
+    _check(lib().bpdq_gate_up_swiglu(gate._h, up._h, x_ptr, h_ptr, M, stream))
+
+
 def bpdq_linear_noalloc(blob_ptr: int, out: int, in_: int, K: int, group: int, x_ptr: int, y_ptr: int, M: int,
                         stream: int = 0) -> None:
     """Look-up-table kernel on a caller-owned device blob; uses the library's static scratch, allocates nothing."""
@@ -195,6 +203,24 @@ class Handle:
 
     def bpdq_set_few_max_m(self, m: int) -> None:
         _check(lib().bpdq_set_few_max_m(self._h, m))
+
+    def bpdq_set_input_permutation(self, perm) -> None:
+        if perm is None:
+            _check(lib().bpdq_set_input_permutation(self._h, None))
+        else:
+            perm = np.ascontiguousarray(perm, dtype=np.int32)
+            if perm.shape != (self.in_,):
+                raise ValueError("perm must have one entry per input channel")
+            _check(lib().bpdq_set_input_permutation(self._h, _np_ptr(perm)))
+
+    def bpdq_set_bias(self, bias_bits) -> None:
+        if bias_bits is None:
+            _check(lib().bpdq_set_bias(self._h, None))
+        else:
+            bias_bits = np.ascontiguousarray(bias_bits, dtype=np.uint16)
+            if bias_bits.shape != (self.out,):
+                raise ValueError("bias must have one entry per output row")
+            _check(lib().bpdq_set_bias(self._h, _np_ptr(bias_bits)))
 
     def bpdq_read_blob(self) -> np.ndarray:
         blob = np.empty(self.packed_bytes, dtype=np.uint8)

@@ -5,6 +5,9 @@
 #include <new>
 
 #include "bpdq_internal.h"
+#include "bpdq_finish.cuh"
+
+#include <cuda_fp16.h>
 
 using namespace bpdq;
 
@@ -25,6 +28,9 @@ void free_handle(bpdq_handle_s* h) {
     if (h->d_xstage) cudaFree(h->d_xstage);
     if (h->d_ystage) cudaFree(h->d_ystage);
     if (h->d_few_maps) cudaFree(h->d_few_maps);
+    if (h->d_perm) cudaFree(h->d_perm);
+    if (h->d_xperm) cudaFree(h->d_xperm);
+    if (h->d_bias) cudaFree(h->d_bias);
     delete h;
 }
 
@@ -46,6 +52,27 @@ __global__ void gather_kernel(const __grid_constant__ GatherParams p) {
         while (i >= p.end16[k]) ++k;
         const unsigned j = i - (k ? p.end16[k - 1] : 0u);
         p.dst[k][j] = p.src[k][j];
+    }
+}
+
+// Activations in stored-column order: dst[m][j] = src[m][perm[j]], eight columns (sixteen bytes) per thread.
+__global__ void gather_columns_kernel(const __half* __restrict__ src, const int* __restrict__ perm, __half* __restrict__ dst,
+                                      int M, int in) {
+    const int chunks = in / 8;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < (long long)M * chunks; i += (long long)gridDim.x * blockDim.x) {
+        const int m = (int)(i / chunks), c = (int)(i % chunks);
+        const int4 p0 = *reinterpret_cast<const int4*>(perm + c * 8), p1 = *reinterpret_cast<const int4*>(perm + c * 8 + 4);
+        const __half* row = src + (size_t)m * in;
+        __align__(16) __half v[8] = {row[p0.x], row[p0.y], row[p0.z], row[p0.w], row[p1.x], row[p1.y], row[p1.z], row[p1.w]};
+        *reinterpret_cast<uint4*>(dst + (size_t)m * in + c * 8) = *reinterpret_cast<const uint4*>(v);
+    }
+}
+
+// h = silu(gate) * up on rounded binary16 inputs (the many-token path of bpdq_gate_up_swiglu), two values per thread.
+__global__ void swiglu_kernel(const __half2* __restrict__ gate, const __half2* __restrict__ up, __half2* __restrict__ hout, size_t n2) {
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n2; i += (size_t)gridDim.x * blockDim.x) {
+        const float2 g = __half22float2(gate[i]), u = __half22float2(up[i]);
+        hout[i] = __floats2half2_rn(bpdq::silu_f32(g.x) * u.x, bpdq::silu_f32(g.y) * u.y);
     }
 }
 
@@ -199,6 +226,12 @@ extern "C" int bpdq_linear_ex(bpdq_handle_t h, const void* x, void* y, int M, in
         else if (gm) kernel = BPDQ_KERNEL_GEMM;
         else kernel = BPDQ_KERNEL_GEMV_SIMPLE;
     }
+    if (h->d_perm && kernel != BPDQ_KERNEL_GEMV) {
+        // only the look-up-table kernel reads x through the permutation; the others get a gathered copy
+        if (x == h->d_xperm) return set_error(BPDQ_ERR_INVALID, "bpdq_linear: x aliases the handle's gather buffer");
+        if (const int rc = launch_gather_columns(h, x, M, s); rc != BPDQ_OK) return rc;
+        x = h->d_xperm;
+    }
     switch (kernel) {
         case BPDQ_KERNEL_GEMV:
             if (M > BPDQ_GEMV_MAX_M)
@@ -235,7 +268,17 @@ extern "C" int bpdq_linear_batch(const bpdq_handle_t* hs, const void* const* xs,
     for (int k = 0; few && k < n; ++k)
         few = hs[k]->d_few_maps && gemv_mma_supported(hs[k]->out, hs[k]->in, hs[k]->K, hs[k]->group) &&
               (size_t)M * hs[k]->out * sizeof(float) <= hs[k]->ws_bytes;
-    if (few) return launch_gemv_mma_batch(hs, xs, ys, n, M, static_cast<cudaStream_t>(stream));
+    if (few) {
+        const void* xg[BPDQ_BATCH_MAX];
+        for (int k = 0; k < n; ++k) {
+            xg[k] = xs[k];
+            if (hs[k]->d_perm) {
+                if (const int rc = launch_gather_columns(hs[k], xs[k], M, static_cast<cudaStream_t>(stream)); rc != BPDQ_OK) return rc;
+                xg[k] = hs[k]->d_xperm;
+            }
+        }
+        return launch_gemv_mma_batch(hs, xg, ys, n, M, static_cast<cudaStream_t>(stream));
+    }
     return launch_gemv_batch(hs, xs, ys, n, M, static_cast<cudaStream_t>(stream));
 }
 
@@ -363,4 +406,122 @@ extern "C" int bpdq_launch_count(bpdq_handle_t h, uint64_t* count) {
     if (!h || !count) return set_error(BPDQ_ERR_INVALID, "bpdq_launch_count: null pointer");
     *count = h->launches;
     return BPDQ_OK;
+}
+
+namespace bpdq {
+
+int launch_gather_columns(bpdq_handle_s* h, const void* x, int M, cudaStream_t stream) {
+    const long long items = (long long)M * (h->in / 8);
+    long long blocks = (items + 255) / 256;
+    if (blocks > 4LL * h->sm_count) blocks = 4LL * h->sm_count;
+    gather_columns_kernel<<<(unsigned)blocks, 256, 0, stream>>>(static_cast<const __half*>(x), h->d_perm, static_cast<__half*>(h->d_xperm), M, h->in);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return set_error(BPDQ_ERR_CUDA, "gather launch: %s", cudaGetErrorString(e));
+    h->launches += 1;
+    return BPDQ_OK;
+}
+
+int launch_swiglu(const void* gate, const void* up, void* hout, size_t n, cudaStream_t stream) {
+    const size_t n2 = n / 2;                                      // out is a multiple of 16: an even count
+    size_t blocks = (n2 + 255) / 256;
+    if (blocks > 1184) blocks = 1184;
+    swiglu_kernel<<<(unsigned)blocks, 256, 0, stream>>>(static_cast<const __half2*>(gate), static_cast<const __half2*>(up), static_cast<__half2*>(hout), n2);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return set_error(BPDQ_ERR_CUDA, "gated unit launch: %s", cudaGetErrorString(e));
+    return BPDQ_OK;
+}
+
+}  // namespace bpdq
+
+extern "C" int bpdq_set_input_permutation(bpdq_handle_t h, const int32_t* perm) {
+    if (!h) return set_error(BPDQ_ERR_INVALID, "bpdq_set_input_permutation: null handle");
+    if (const int rc = check_device(h, "bpdq_set_input_permutation"); rc != BPDQ_OK) return rc;
+    cudaError_t e = cudaDeviceSynchronize();                      // nothing in flight may still read the old permutation
+    if (e != cudaSuccess) return cuda_fail("bpdq_set_input_permutation: synchronize", e);
+    if (!perm) {
+        if (h->d_perm) cudaFree(h->d_perm);
+        if (h->d_xperm) cudaFree(h->d_xperm);
+        h->d_perm = nullptr; h->d_xperm = nullptr;
+        return BPDQ_OK;
+    }
+    {
+        unsigned char* seen = new (std::nothrow) unsigned char[h->in]();
+        if (!seen) return set_error(BPDQ_ERR_ALLOC, "bpdq_set_input_permutation: host allocation failed");
+        bool ok = true;
+        for (int j = 0; j < h->in && ok; ++j) {
+            ok = perm[j] >= 0 && perm[j] < h->in && !seen[perm[j]];
+            if (ok) seen[perm[j]] = 1;
+        }
+        delete[] seen;
+        if (!ok) return set_error(BPDQ_ERR_INVALID, "bpdq_set_input_permutation: not a permutation of 0..%d", h->in - 1);
+    }
+    if (!h->d_perm && (e = cudaMalloc(&h->d_perm, (size_t)h->in * sizeof(int))) != cudaSuccess) {
+        h->d_perm = nullptr;
+        return set_error(BPDQ_ERR_ALLOC, "bpdq_set_input_permutation: cudaMalloc failed (%s)", cudaGetErrorString(e));
+    }
+    if (!h->d_xperm && (e = cudaMalloc(&h->d_xperm, (size_t)h->max_M * h->in * 2)) != cudaSuccess) {
+        cudaFree(h->d_perm);
+        h->d_perm = nullptr; h->d_xperm = nullptr;
+        return set_error(BPDQ_ERR_ALLOC, "bpdq_set_input_permutation: cudaMalloc failed (%s)", cudaGetErrorString(e));
+    }
+    e = cudaMemcpy(h->d_perm, perm, (size_t)h->in * sizeof(int), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) return cuda_fail("bpdq_set_input_permutation: copy", e);
+    return BPDQ_OK;
+}
+
+extern "C" int bpdq_set_bias(bpdq_handle_t h, const uint16_t* bias) {
+    if (!h) return set_error(BPDQ_ERR_INVALID, "bpdq_set_bias: null handle");
+    if (const int rc = check_device(h, "bpdq_set_bias"); rc != BPDQ_OK) return rc;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail("bpdq_set_bias: synchronize", e);
+    if (!bias) {
+        if (h->d_bias) cudaFree(h->d_bias);
+        h->d_bias = nullptr;
+        return BPDQ_OK;
+    }
+    if (!h->d_bias && (e = cudaMalloc(&h->d_bias, (size_t)h->out * 2)) != cudaSuccess) {
+        h->d_bias = nullptr;
+        return set_error(BPDQ_ERR_ALLOC, "bpdq_set_bias: cudaMalloc failed (%s)", cudaGetErrorString(e));
+    }
+    e = cudaMemcpy(h->d_bias, bias, (size_t)h->out * 2, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) return cuda_fail("bpdq_set_bias: copy", e);
+    return BPDQ_OK;
+}
+
+extern "C" int bpdq_gate_up_swiglu(bpdq_handle_t hg, bpdq_handle_t hu, const void* x, void* hout, int M, void* stream) {
+    if (!hg || !hu) return set_error(BPDQ_ERR_INVALID, "bpdq_gate_up_swiglu: null handle");
+    if (hg == hu) return set_error(BPDQ_ERR_INVALID, "bpdq_gate_up_swiglu: gate and up are the same handle");
+    if (hg->out != hu->out || hg->in != hu->in || hg->K != hu->K || hg->device != hu->device)
+        return set_error(BPDQ_ERR_INVALID, "bpdq_gate_up_swiglu: gate and up differ in shape, K or device");
+    if (M < 0 || M > hg->max_M || M > hu->max_M) return set_error(BPDQ_ERR_INVALID, "bpdq_gate_up_swiglu: M=%d outside [0, max_M]", M);
+    if (M == 0) return BPDQ_OK;
+    if (!x || !hout || !aligned16(x) || !aligned16(hout))
+        return set_error(BPDQ_ERR_INVALID, "bpdq_gate_up_swiglu: x and h must be non-null and 16-byte aligned");
+    if (const int rc = check_device(hg, "bpdq_gate_up_swiglu"); rc != BPDQ_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    bpdq_handle_s* hs[2] = {hg, hu};
+    const bool same_g64 = (hg->group == 64) == (hu->group == 64);
+    const bool lut = same_g64 && M <= hg->gemv_max_m && M <= BPDQ_GEMV_MAX_M && gemv_supported(hg->out, hg->in, hg->K, hg->group) &&
+                     gemv_supported(hu->out, hu->in, hu->K, hu->group);
+    bool few = same_g64 && !lut && M <= hg->few_max_m && M <= BPDQ_FEW_MAX_M && hg->d_few_maps && hu->d_few_maps &&
+               (size_t)M * hg->out * sizeof(float) <= hg->ws_bytes && (size_t)M * hu->out * sizeof(float) <= hu->ws_bytes;
+    if (lut || few) {
+        // one launch over both linears; the kernel that completes a block of rows applies the unit
+        const void* xs[2] = {x, x};
+        if (few) {                                                 // this kernel does not read through a permutation: gather first
+            for (int k = 0; k < 2; ++k) {
+                if (hs[k]->d_perm) {
+                    if (const int rc = launch_gather_columns(hs[k], x, M, s); rc != BPDQ_OK) return rc;
+                    xs[k] = hs[k]->d_xperm;
+                }
+            }
+        }
+        void* ys[2] = {hout, hout};
+        return lut ? launch_gemv_batch(hs, xs, ys, 2, M, s, true) : launch_gemv_mma_batch(hs, xs, ys, 2, M, s, true);
+    }
+    // many tokens: both projections through the dispatcher into the handles' own output buffers, then the unit
+    for (int k = 0; k < 2; ++k)
+        if (const int rc = bpdq_linear_ex(hs[k], x, hs[k]->d_ystage, M, BPDQ_KERNEL_AUTO, stream); rc != BPDQ_OK) return rc;
+    hg->launches += 1;
+    return launch_swiglu(hg->d_ystage, hu->d_ystage, hout, (size_t)M * hg->out, s);
 }

@@ -85,6 +85,7 @@ struct GemmParams {
     int kb_per;               // stages per CTA (even: a 128-column block is never cut)
     float* ws;                // [M][out] binary32, zero between calls (only used when gridDim.z > 1)
     unsigned* counters;       // one arrival counter per 128-row tile, zero between calls
+    const __half* bias;       // binary16 [out] added before the rounding, or null
 };
 
 // ---- PTX wrappers (mbarrier and TMA ones live in bpdq_tma.cuh) ------------------------------
@@ -366,12 +367,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
                     for (int j = 0; j < 16; ++j) acc[j] += __uint_as_float(v[j]);
                 }
                 if (row_ok) {
+                    const float br = (p.bias && gridDim.z == 1) ? __half2float(p.bias[r]) : 0.f;   // a shared tile gets it when it is completed
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const int t = tok0 + c0 + j;
                         if (t < p.M) {
                             if (gridDim.z > 1) atomicAdd(p.ws + (size_t)t * p.out + r, acc[j]);
-                            else p.y[(size_t)t * p.out + r] = __float2half_rn(acc[j]);
+                            else p.y[(size_t)t * p.out + r] = __float2half_rn(acc[j] + br);
                         }
                     }
                 }
@@ -401,7 +403,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
                 const int t = tok0 + idx / BM, r = row0 + idx % BM;
                 if (r < p.out) {
                     float* src = p.ws + (size_t)t * p.out + r;
-                    p.y[(size_t)t * p.out + r] = __float2half_rn(__ldcg(src));
+                    p.y[(size_t)t * p.out + r] = __float2half_rn(__ldcg(src) + (p.bias ? __half2float(p.bias[r]) : 0.f));
                     __stcg(src, 0.f);
                 }
             }
@@ -616,10 +618,11 @@ gemm_persistent_kernel(const __grid_constant__ CUtensorMap x_map, const GemmPara
                 tmem_ld16(taddr + (unsigned)c0, v);
                 tmem_ld_wait();
                 if (row_ok) {
+                    const float br = p.bias ? __half2float(p.bias[r]) : 0.f;
 #pragma unroll
                     for (int jj = 0; jj < 16; ++jj) {
                         const int t = tok0 + c0 + jj;
-                        if (t < p.M) p.y[(size_t)t * p.out + r] = __float2half_rn(__uint_as_float(v[jj]));
+                        if (t < p.M) p.y[(size_t)t * p.out + r] = __float2half_rn(__uint_as_float(v[jj]) + br);
                     }
                 }
             }
@@ -678,7 +681,7 @@ int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t st
     GemmParams p;
     p.blob = h->d_blob; p.planes_bytes = h->planes_bytes; p.y = static_cast<__half*>(y); p.status = h->d_status;
     p.out = h->out; p.in = h->in; p.group = h->group; p.M = M;
-    p.ws = h->d_ws; p.counters = h->d_counters;
+    p.ws = h->d_ws; p.counters = h->d_counters; p.bias = static_cast<const __half*>(h->d_bias);
     dim3 grid((h->out + BM - 1) / BM, (M + BN - 1) / BN);
     const int nkb = h->in / BK;
     p.kb_per = nkb;
@@ -720,7 +723,7 @@ int launch_persistent(bpdq_handle_s* h, const void* x, void* y, int M, cudaStrea
     GemmParams p;
     p.blob = h->d_blob; p.planes_bytes = h->planes_bytes; p.y = static_cast<__half*>(y); p.status = h->d_status;
     p.out = h->out; p.in = h->in; p.group = h->group; p.M = M;
-    p.ws = h->d_ws; p.counters = h->d_counters; p.kb_per = h->in / BK;
+    p.ws = h->d_ws; p.counters = h->d_counters; p.kb_per = h->in / BK; p.bias = static_cast<const __half*>(h->d_bias);
     const long long ntiles = (long long)((h->out + BM - 1) / BM) * ((M + kPersistBN - 1) / kPersistBN);
     const int grid = ntiles < h->sm_count ? (int)ntiles : h->sm_count;
     gemm_persistent_kernel<K><<<grid, kPersistThreads, C::kSmemBytes, stream>>>(map, p);

@@ -29,6 +29,7 @@
 // Algorithmic HBM bytes per weight: K/8 + 2(K+1)/g.
 #include "bpdq_internal.h"
 #include "bpdq_partition.h"
+#include "bpdq_finish.cuh"
 
 #include <cuda_fp16.h>
 
@@ -51,6 +52,14 @@ struct GemvLinear {
     __half* y;                // [MT][out]
     float* ws;                // [MT][out] binary32 row sums, zero between calls
     unsigned* counters;       // [ceil(out/16 / kChunkRgs)] arrival counters, zero between calls
+    // completion: a finished chunk is converted from conv_a (this linear's sums) or, for a (gate, up) pair, from
+    // conv_a = gate's and conv_b = up's sums as silu(a) * b; the pair shares gate's counters and both count into them
+    float* conv_a;
+    float* conv_b;            // null unless paired
+    const __half* bias_a;     // null: none
+    const __half* bias_b;
+    int target_mul;           // 1, or 2 for a pair
+    const int* perm;          // null: identity; else stored column j multiplies x[perm[j]]
     int out, in, group;
     int nblocks, nslices, nrg;
     int task_begin;           // first task of this linear in the concatenated task space
@@ -94,6 +103,11 @@ __device__ __forceinline__ uint4 ldg_stream16(const uint8_t* p) {
 __device__ __forceinline__ unsigned ldg_x4(const void* p) {
     unsigned v;
     asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned short ldg_x2(const void* p) {
+    unsigned short v;
+    asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(v) : "l"(p) : "memory");
     return v;
 }
 __device__ __forceinline__ unsigned ldg_stream4(const uint8_t* p) {
@@ -218,7 +232,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                 const int lo = max(rg_begin, ck * kChunkRgs), hi = min(rg_end, (ck + 1) * kChunkRgs);
                 const int size = min(L.nrg, (ck + 1) * kChunkRgs) - ck * kChunkRgs;
                 const unsigned before = atomicAdd(&L.counters[ck], (unsigned)(hi - lo));
-                if (before + (unsigned)(hi - lo) == (unsigned)(size * L.nslices)) {
+                if (before + (unsigned)(hi - lo) == (unsigned)(size * L.nslices * L.target_mul)) {
                     L.counters[ck] = 0u;
                     done[atomicAdd(ndone, 1)] = ck;
                 }
@@ -232,8 +246,9 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                 constexpr int kQuads = kChunkRgs * 16 / 4, kAhead = 4;
                 const int nitems = nd * MT * kQuads;
                 for (int i0 = tid; i0 < nitems; i0 += kThreads * kAhead) {
-                    float4 v[kAhead];
+                    float4 v[kAhead], vb[kAhead];
                     size_t at[kAhead];
+                    int row[kAhead];
                     bool live[kAhead];
 #pragma unroll
                     for (int u = 0; u < kAhead; ++u) {
@@ -245,20 +260,24 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                             const int r = ckd * kChunkRgs * 16 + (rem % kQuads) * 4;
                             if (r < L.out) {                  // out is a multiple of 16: a quad is inside or outside as a whole
                                 live[u] = true;
+                                row[u] = r;
                                 at[u] = (size_t)(rem / kQuads) * L.out + r;
-                                v[u] = __ldcg(reinterpret_cast<const float4*>(L.ws + at[u]));
+                                v[u] = __ldcg(reinterpret_cast<const float4*>(L.conv_a + at[u]));
+                                if (L.conv_b) vb[u] = __ldcg(reinterpret_cast<const float4*>(L.conv_b + at[u]));
                             }
                         }
                     }
 #pragma unroll
                     for (int u = 0; u < kAhead; ++u) {
                         if (live[u]) {
+                            bpdq::finish_quad(v[u], vb[u], L.bias_a, L.bias_b, L.conv_b != nullptr, row[u]);
+                            if (L.conv_b) __stcg(reinterpret_cast<float4*>(L.conv_b + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
                             const __half2 h01 = __floats2half2_rn(v[u].x, v[u].y), h23 = __floats2half2_rn(v[u].z, v[u].w);
                             uint2 o;
                             o.x = *reinterpret_cast<const unsigned*>(&h01);
                             o.y = *reinterpret_cast<const unsigned*>(&h23);
                             *reinterpret_cast<uint2*>(L.y + at[u]) = o;
-                            __stcg(reinterpret_cast<float4*>(L.ws + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
+                            __stcg(reinterpret_cast<float4*>(L.conv_a + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
                         }
                     }
                 }
@@ -350,7 +369,10 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
         for (int m = 0; m < MT; ++m)
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                xraw[m][u] = col < L.in ? ldg_x4(L.x + (size_t)m * L.in + col + 8 * u) : 0u;
+                xraw[m][u] = col >= L.in ? 0u
+                             : !L.perm   ? ldg_x4(L.x + (size_t)m * L.in + col + 8 * u)
+                                         : (unsigned)ldg_x2(L.x + (size_t)m * L.in + __ldg(L.perm + col + 8 * u)) |
+                                               ((unsigned)ldg_x2(L.x + (size_t)m * L.in + __ldg(L.perm + col + 8 * u + 1)) << 16);
         if (!early) {
 #pragma unroll
             for (int d = 0; d < D; ++d)
@@ -604,6 +626,10 @@ void fill_linear(GemvLinear& L, const bpdq_handle_s* h) {
     L.blob_bytes = h->blob_bytes;
     L.ws = h->d_ws;
     L.counters = h->d_counters;
+    L.conv_a = h->d_ws; L.conv_b = nullptr;
+    L.bias_a = static_cast<const __half*>(h->d_bias); L.bias_b = nullptr;
+    L.target_mul = 1;
+    L.perm = h->d_perm;
     L.out = h->out; L.in = h->in; L.group = h->group;
     L.nblocks = h->in / 128;
     L.nslices = (L.nblocks + kSliceBlocks - 1) / kSliceBlocks;
@@ -620,7 +646,7 @@ int launch_k(bpdq_handle_s* const* hs, GemvParams p, const void* const* xs, void
         if (mt > kMaxMT) mt = kMaxMT;
         for (int k = 0; k < p.n; ++k) {
             p.lin[k].x = static_cast<const __half*>(xs[k]) + (size_t)m0 * hs[k]->in;
-            p.lin[k].y = static_cast<__half*>(ys[k]) + (size_t)m0 * hs[k]->out;
+            p.lin[k].y = static_cast<__half*>(ys[p.lin[k].target_mul == 2 ? 0 : k]) + (size_t)m0 * hs[k]->out;   // a pair writes one output
         }
         const int rc = (mt == 1) ? launch_one<K, 1>(hs[0], p, stream) : launch_one<K, 2>(hs[0], p, stream);
         if (rc != BPDQ_OK) return rc;
@@ -648,8 +674,9 @@ size_t gemv_workspace_bytes(int out, int, int, int, int max_M, int) {
 
 size_t gemv_counter_count(int out) { return ((size_t)out / 16 + kChunkRgs - 1) / kChunkRgs; }
 
-int launch_gemv_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream) {
+int launch_gemv_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream, bool pair) {
     if (n < 1 || n > kMaxBatch) return set_error(BPDQ_ERR_INVALID, "gemv: %d linears in one launch (1..%d)", n, kMaxBatch);
+    if (pair && (n != 2 || hs[0]->out != hs[1]->out)) return set_error(BPDQ_ERR_INVALID, "gemv: a (gate, up) pair is two linears with the same rows");
     GemvParams p;
     p.n = n;
     p.status = hs[0]->d_status;
@@ -660,6 +687,15 @@ int launch_gemv_batch(bpdq_handle_s* const* hs, const void* const* xs, void* con
             return set_error(BPDQ_ERR_INVALID, "gemv: linears of one launch must all have group 64 or none of them");
         fill_linear(p.lin[k], hs[k]);
         if (hs[k]->caller_blob) p.early_weights = 0;
+    }
+    if (pair) {                                          // both count into gate's counters; whoever completes a chunk converts both sums
+        for (int k = 0; k < 2; ++k) {
+            GemvLinear& L = p.lin[k];
+            L.counters = hs[0]->d_counters;
+            L.conv_a = hs[0]->d_ws; L.conv_b = hs[1]->d_ws;
+            L.bias_a = static_cast<const __half*>(hs[0]->d_bias); L.bias_b = static_cast<const __half*>(hs[1]->d_bias);
+            L.target_mul = 2;
+        }
     }
     switch (hs[0]->K) {
         case 1: return launch_k<1>(hs, p, xs, ys, M, stream);

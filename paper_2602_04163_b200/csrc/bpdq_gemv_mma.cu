@@ -37,6 +37,7 @@
 #include "bpdq_decode.cuh"
 #include "bpdq_partition.h"
 #include "bpdq_tma.cuh"
+#include "bpdq_finish.cuh"
 
 #include <cuda_fp16.h>
 #include <type_traits>
@@ -59,6 +60,13 @@ struct MmaLinear {
     __half* y;                // [M][out]
     float* ws;                // [M][out] binary32, zero between calls
     unsigned* counters;       // one per 128 rows, zero between calls
+    // completion (as in the look-up-table kernel): a finished chunk is converted from conv_a, or for a (gate, up)
+    // pair as silu(conv_a) * conv_b; the pair shares gate's counters and both count into them
+    float* conv_a;
+    float* conv_b;            // null unless paired
+    const __half* bias_a;     // null: none
+    const __half* bias_b;
+    int target_mul;           // 1, or 2 for a pair
     int out, in, group;
     int gsh;                  // coefficient group of a half block: (2 b + half) >> gsh
     int nblocks, nslices;     // 128-column blocks, 512-column slices
@@ -179,7 +187,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_mma_kernel(const __grid_consta
                 const int size = min(L.nrg, (ck + 1) * kChunkRgs) - ck * kChunkRgs;
                 const unsigned mine = (unsigned)((hi - lo) * nsl);
                 const unsigned before = atomicAdd(&L.counters[ck], mine);
-                if (before + mine == (unsigned)(size * L.nslices)) {
+                if (before + mine == (unsigned)(size * L.nslices * L.target_mul)) {
                     L.counters[ck] = 0u;
                     done[atomicAdd(ndone, 1)] = ck;
                 }
@@ -191,8 +199,9 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_mma_kernel(const __grid_consta
                 constexpr int kQuads = kChunkRows / 4, kAhead = 4;
                 const int nitems = nd * p.M * kQuads;
                 for (int i0 = tid; i0 < nitems; i0 += kThreads * kAhead) {
-                    float4 v[kAhead];
+                    float4 v[kAhead], vb[kAhead];
                     size_t at[kAhead];
+                    int row[kAhead];
                     bool live[kAhead];
 #pragma unroll
                     for (int u = 0; u < kAhead; ++u) {
@@ -204,20 +213,24 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_mma_kernel(const __grid_consta
                             const int r = ckd * kChunkRows + (rem % kQuads) * 4;
                             if (r < L.out) {
                                 live[u] = true;
+                                row[u] = r;
                                 at[u] = (size_t)(rem / kQuads) * L.out + r;
-                                v[u] = __ldcg(reinterpret_cast<const float4*>(L.ws + at[u]));
+                                v[u] = __ldcg(reinterpret_cast<const float4*>(L.conv_a + at[u]));
+                                if (L.conv_b) vb[u] = __ldcg(reinterpret_cast<const float4*>(L.conv_b + at[u]));
                             }
                         }
                     }
 #pragma unroll
                     for (int u = 0; u < kAhead; ++u) {
                         if (live[u]) {
+                            bpdq::finish_quad(v[u], vb[u], L.bias_a, L.bias_b, L.conv_b != nullptr, row[u]);
+                            if (L.conv_b) __stcg(reinterpret_cast<float4*>(L.conv_b + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
                             const __half2 h01 = __floats2half2_rn(v[u].x, v[u].y), h23 = __floats2half2_rn(v[u].z, v[u].w);
                             uint2 o;
                             o.x = *reinterpret_cast<const unsigned*>(&h01);
                             o.y = *reinterpret_cast<const unsigned*>(&h23);
                             *reinterpret_cast<uint2*>(L.y + at[u]) = o;
-                            __stcg(reinterpret_cast<float4*>(L.ws + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
+                            __stcg(reinterpret_cast<float4*>(L.conv_a + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
                         }
                     }
                 }
@@ -563,8 +576,9 @@ int few_prepare(bpdq_handle_s* h) {
     return BPDQ_OK;
 }
 
-int launch_gemv_mma_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream) {
+int launch_gemv_mma_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream, bool pair) {
     if (n < 1 || n > kMaxBatch) return set_error(BPDQ_ERR_INVALID, "gemv_mma: %d linears in one launch (1..%d)", n, kMaxBatch);
+    if (pair && (n != 2 || hs[0]->out != hs[1]->out)) return set_error(BPDQ_ERR_INVALID, "gemv_mma: a (gate, up) pair is two linears with the same rows");
     if (M < 1 || M > BPDQ_FEW_MAX_M) return set_error(BPDQ_ERR_INVALID, "gemv_mma: M=%d outside [1, %d]", M, BPDQ_FEW_MAX_M);
     MmaParams p;
     p.n = n; p.M = M;
@@ -581,8 +595,12 @@ int launch_gemv_mma_batch(bpdq_handle_s* const* hs, const void* const* xs, void*
             return set_error(BPDQ_ERR_INVALID, "gemv_mma: M=%d exceeds the workspace of linear %d (max_M=%d)", M, k, h->max_M);
         MmaLinear& L = p.lin[k];
         L.maps = static_cast<const CUtensorMap*>(h->d_few_maps);
-        L.x = static_cast<const __half*>(xs[k]); L.y = static_cast<__half*>(ys[k]);
-        L.ws = h->d_ws; L.counters = h->d_counters;
+        L.x = static_cast<const __half*>(xs[k]); L.y = static_cast<__half*>(ys[pair ? 0 : k]);
+        L.ws = h->d_ws; L.counters = pair ? hs[0]->d_counters : h->d_counters;
+        L.conv_a = pair ? hs[0]->d_ws : h->d_ws; L.conv_b = pair ? hs[1]->d_ws : nullptr;
+        L.bias_a = static_cast<const __half*>(pair ? hs[0]->d_bias : h->d_bias);
+        L.bias_b = pair ? static_cast<const __half*>(hs[1]->d_bias) : nullptr;
+        L.target_mul = pair ? 2 : 1;
         L.out = h->out; L.in = h->in; L.group = h->group;
         L.gsh = h->group == 64 ? 0 : (h->group == 128 ? 1 : 2);
         L.nblocks = h->in / 128;

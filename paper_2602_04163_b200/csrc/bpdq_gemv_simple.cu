@@ -13,7 +13,7 @@ namespace {
 template <int K>
 __global__ void __launch_bounds__(128)
 gemv_simple_kernel(const uint8_t* __restrict__ blob, size_t planes_bytes, const __half* __restrict__ x,
-                   __half* __restrict__ y, int out, int in, int group) {
+                   __half* __restrict__ y, int out, int in, int group, const __half* __restrict__ bias) {
     constexpr int NC = 1 << K;
     const int r = blockIdx.x * 128 + threadIdx.x;
     const int m = blockIdx.y;
@@ -62,7 +62,7 @@ gemv_simple_kernel(const uint8_t* __restrict__ blob, size_t planes_bytes, const 
             }
         }
     }
-    y[(size_t)m * out + r] = __float2half_rn(acc);
+    y[(size_t)m * out + r] = __float2half_rn(acc + (bias ? __half2float(bias[r]) : 0.f));
 }
 
 }  // namespace
@@ -74,10 +74,10 @@ int launch_gemv_simple(bpdq_handle_s* h, const void* x, void* y, int M, cudaStre
     const __half* xp = static_cast<const __half*>(x);
     __half* yp = static_cast<__half*>(y);
     switch (h->K) {
-        case 1: gemv_simple_kernel<1><<<grid, block, 0, stream>>>(h->d_blob, h->planes_bytes, xp, yp, h->out, h->in, h->group); break;
-        case 2: gemv_simple_kernel<2><<<grid, block, 0, stream>>>(h->d_blob, h->planes_bytes, xp, yp, h->out, h->in, h->group); break;
-        case 3: gemv_simple_kernel<3><<<grid, block, 0, stream>>>(h->d_blob, h->planes_bytes, xp, yp, h->out, h->in, h->group); break;
-        case 4: gemv_simple_kernel<4><<<grid, block, 0, stream>>>(h->d_blob, h->planes_bytes, xp, yp, h->out, h->in, h->group); break;
+        case 1: gemv_simple_kernel<1><<<grid, block, 0, stream>>>(h->d_blob, h->planes_bytes, xp, yp, h->out, h->in, h->group, static_cast<const __half*>(h->d_bias)); break;
+        case 2: gemv_simple_kernel<2><<<grid, block, 0, stream>>>(h->d_blob, h->planes_bytes, xp, yp, h->out, h->in, h->group, static_cast<const __half*>(h->d_bias)); break;
+        case 3: gemv_simple_kernel<3><<<grid, block, 0, stream>>>(h->d_blob, h->planes_bytes, xp, yp, h->out, h->in, h->group, static_cast<const __half*>(h->d_bias)); break;
+        case 4: gemv_simple_kernel<4><<<grid, block, 0, stream>>>(h->d_blob, h->planes_bytes, xp, yp, h->out, h->in, h->group, static_cast<const __half*>(h->d_bias)); break;
         default: return set_error(BPDQ_ERR_UNSUPPORTED, "gemv_simple: K=%d", h->K);
     }
     h->launches += 1;

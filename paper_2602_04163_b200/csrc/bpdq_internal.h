@@ -80,6 +80,9 @@ struct bpdq_handle_s {
     uint64_t launches;
     int few_max_m;            // largest M the dispatcher sends to the few-token kernel
     void* d_few_maps;         // device copy of the few-token kernel's two tensor maps (null: not available)
+    int* d_perm;              // input-channel permutation: stored column j multiplies x[perm[j]] (null: identity)
+    void* d_xperm;            // [max_M][in] gathered activations for the kernels that do not fold the permutation into their loads
+    void* d_bias;             // binary16 [out], added to every output row before the rounding (null: none)
     // Tensor maps of the blob for the tensor-core kernel (planes, coefficients), encoded at the first launch.
     alignas(64) unsigned char gemm_maps[2][128];
     int gemm_maps_ready;
@@ -92,10 +95,12 @@ int launch_fill(bpdq_handle_s* h, uint64_t seed, cudaStream_t stream);
 int launch_dequant(bpdq_handle_s* h, void* w, cudaStream_t stream);
 int launch_gemv_simple(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
 int launch_gemv(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
-int launch_gemv_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream);
+int launch_gemv_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream, bool pair = false);
 int launch_gemm(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
+int launch_gather_columns(bpdq_handle_s* h, const void* x, int M, cudaStream_t stream);   // x[m][perm[j]] -> d_xperm[m][j]
+int launch_swiglu(const void* gate, const void* up, void* hout, size_t n, cudaStream_t stream);
 int launch_gemv_mma(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
-int launch_gemv_mma_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream);
+int launch_gemv_mma_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream, bool pair = false);
 bool gemv_mma_supported(int out, int in, int K, int group);
 int few_prepare(bpdq_handle_s* h);
 size_t gemv_workspace_bytes(int out, int in, int K, int group, int max_M, int sm_count);
