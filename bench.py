@@ -632,6 +632,81 @@ def extra_sections(torch, binding, args, peaks, sp, stream):
             h.bpdq_destroy()
         del xs, ys
 
+    # steps around the linears: input-channel permutation and bias on the gate projection (M = 1 and M = 8192), the
+    # gated unit over (gate, up) as one call, and planes made by the data-free producer instead of random ones
+    for K in (2,):
+        o, i = 29568, 8192
+        hs3 = [binding.Handle(o, i, K, GROUP, None, 1400 + c, 8192) for c in range(3)]
+        rec = {}
+        perm = np.concatenate([G_ * GROUP + np.random.default_rng(G_).permutation(GROUP) for G_ in np.random.default_rng(1).permutation(i // GROUP)]).astype(np.int32)
+        for M in (1, 8, 8192):
+            x = xt(M, i)
+            y = torch.empty((M, o), dtype=torch.float16, device="cuda")
+            n = 30 if M < 100 else 3
+
+            def run_lin():
+                for k in range(n):
+                    hs3[k % 3].bpdq_linear(x.data_ptr(), y.data_ptr(), M, sp)
+            run_lin()
+            base = event_time_ms(torch, run_lin, stream) / n
+            for h in hs3:
+                h.bpdq_set_input_permutation(perm)
+            run_lin()
+            with_perm = event_time_ms(torch, run_lin, stream) / n
+            for h in hs3:
+                h.bpdq_set_input_permutation(None)
+                h.bpdq_set_bias(np.zeros(o, dtype=np.uint16))
+            run_lin()
+            with_bias = event_time_ms(torch, run_lin, stream) / n
+            for h in hs3:
+                h.bpdq_set_bias(None)
+            rec[f"M{M}"] = {"us_plain": base * 1e3, "us_with_permutation": with_perm * 1e3, "us_with_bias": with_bias * 1e3}
+        out["gate_K2_permutation_and_bias_cost"] = rec
+        up3 = [binding.Handle(o, i, K, GROUP, None, 1410 + c, 16) for c in range(3)]
+        recs = {}
+        for M in (1, 8):
+            x = xt(M, i)
+            hh = torch.empty((M, o), dtype=torch.float16, device="cuda")
+            n = 30
+
+            def run_unit():
+                for k in range(n):
+                    binding.bpdq_gate_up_swiglu(hs3[k % 3], up3[k % 3], x.data_ptr(), hh.data_ptr(), M, sp)
+            run_unit()
+            ms = event_time_ms(torch, run_unit, stream) / n
+            b = 2 * useful_bytes(o, i, K, GROUP, M) - M * i * 2 - M * o * 2
+            recs[f"M{M}"] = {"us": ms * 1e3, "gbs": b / (ms * 1e-3) / 1e9, "frac_measured": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        out["gate_up_gated_unit_K2"] = recs
+        for h in hs3 + up3:
+            h.bpdq_destroy()
+    # structured planes: a 7B-shaped gate projection quantized by the data-free producer (most significant bits of
+    # Gaussian weights with outliers, fitted coefficients) against the same shape with random planes
+    for K in (2,):
+        o, i = 18944, 3584
+        rng = np.random.default_rng(7)
+        w = rng.normal(0, 0.02, size=(o, i)).astype(np.float32)
+        w[rng.random(w.shape) < 0.002] *= 10.0
+        bits, coef = binding.bpdq_quantize_datafree(w, K, GROUP)
+        blob = binding.bpdq_pack(bits, coef, GROUP)
+        del w, bits, coef
+        copies = 8
+        structured = [binding.Handle(o, i, K, GROUP, blob, 0, 8) for _ in range(copies)]
+        random_ = [binding.Handle(o, i, K, GROUP, None, 1500 + c, 8) for c in range(copies)]
+        rec = {"shape": [o, i], "K": K, "copies_rotated": copies}
+        for M in (1, 8):
+            x = xt(M, i)
+            y = torch.empty((M, o), dtype=torch.float16, device="cuda")
+            n = 80
+            for tag, hl in (("structured", structured), ("random", random_)):
+                def run_s():
+                    for k in range(n):
+                        hl[k % copies].bpdq_linear(x.data_ptr(), y.data_ptr(), M, sp)
+                run_s()
+                rec[f"us_{tag}_M{M}"] = event_time_ms(torch, run_s, stream) / n * 1e3
+        out["structured_planes_7b_gate_K2"] = rec
+        for h in structured + random_:
+            h.bpdq_destroy()
+
     # a decoder layer with a few tokens in flight (M = 4, 8, 16): the grouping a decoder allows, one bpdq_linear_batch
     # call per group (the few-token kernel takes them above two tokens)
     for K in (2, 3):

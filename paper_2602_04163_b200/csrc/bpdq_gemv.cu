@@ -160,7 +160,10 @@ __device__ __forceinline__ float2 unpack2(unsigned long long v) {
     return f;
 }
 
-template <int K, int MT, int D, int W, bool G64>
+// EXT: the launch uses an input permutation, a bias or a (gate, up) pair somewhere.  The plain instantiation carries none of
+// that code: the streaming loop sits at the 128-register cap, and the extra live values cost it spills (5 % of the
+// headline, up to 50 % at g = 64) although they are only used outside the loop.
+template <int K, int MT, int D, int W, bool G64, bool EXT>
 __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_constant__ GemvParams p) {
     constexpr int kThreads = W * 32;
     constexpr int NS = K * MT;                        // look-up streams per step: (plane, token) pairs
@@ -232,7 +235,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                 const int lo = max(rg_begin, ck * kChunkRgs), hi = min(rg_end, (ck + 1) * kChunkRgs);
                 const int size = min(L.nrg, (ck + 1) * kChunkRgs) - ck * kChunkRgs;
                 const unsigned before = atomicAdd(&L.counters[ck], (unsigned)(hi - lo));
-                if (before + (unsigned)(hi - lo) == (unsigned)(size * L.nslices * L.target_mul)) {
+                if (before + (unsigned)(hi - lo) == (unsigned)(size * L.nslices * (EXT ? L.target_mul : 1))) {
                     L.counters[ck] = 0u;
                     done[atomicAdd(ndone, 1)] = ck;
                 }
@@ -262,22 +265,24 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                                 live[u] = true;
                                 row[u] = r;
                                 at[u] = (size_t)(rem / kQuads) * L.out + r;
-                                v[u] = __ldcg(reinterpret_cast<const float4*>(L.conv_a + at[u]));
-                                if (L.conv_b) vb[u] = __ldcg(reinterpret_cast<const float4*>(L.conv_b + at[u]));
+                                v[u] = __ldcg(reinterpret_cast<const float4*>((EXT ? L.conv_a : L.ws) + at[u]));
+                                if (EXT && L.conv_b) vb[u] = __ldcg(reinterpret_cast<const float4*>(L.conv_b + at[u]));
                             }
                         }
                     }
 #pragma unroll
                     for (int u = 0; u < kAhead; ++u) {
                         if (live[u]) {
-                            bpdq::finish_quad(v[u], vb[u], L.bias_a, L.bias_b, L.conv_b != nullptr, row[u]);
-                            if (L.conv_b) __stcg(reinterpret_cast<float4*>(L.conv_b + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
+                            if (EXT) {
+                                bpdq::finish_quad(v[u], vb[u], L.bias_a, L.bias_b, L.conv_b != nullptr, row[u]);
+                                if (L.conv_b) __stcg(reinterpret_cast<float4*>(L.conv_b + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
+                            }
                             const __half2 h01 = __floats2half2_rn(v[u].x, v[u].y), h23 = __floats2half2_rn(v[u].z, v[u].w);
                             uint2 o;
                             o.x = *reinterpret_cast<const unsigned*>(&h01);
                             o.y = *reinterpret_cast<const unsigned*>(&h23);
                             *reinterpret_cast<uint2*>(L.y + at[u]) = o;
-                            __stcg(reinterpret_cast<float4*>(L.conv_a + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
+                            __stcg(reinterpret_cast<float4*>((EXT ? L.conv_a : L.ws) + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
                         }
                     }
                 }
@@ -370,7 +375,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
 #pragma unroll
             for (int u = 0; u < 4; ++u)
                 xraw[m][u] = col >= L.in ? 0u
-                             : !L.perm   ? ldg_x4(L.x + (size_t)m * L.in + col + 8 * u)
+                             : !(EXT && L.perm) ? ldg_x4(L.x + (size_t)m * L.in + col + 8 * u)
                                          : (unsigned)ldg_x2(L.x + (size_t)m * L.in + __ldg(L.perm + col + 8 * u)) |
                                                ((unsigned)ldg_x2(L.x + (size_t)m * L.in + __ldg(L.perm + col + 8 * u + 1)) << 16);
         if (!early) {
@@ -562,13 +567,13 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
     if (pend_li >= 0) hand_over(p.lin[pend_li], pend_begin, pend_end);
 }
 
-template <int K, int MT, int D, int W, bool G64>
+template <int K, int MT, int D, int W, bool G64, bool EXT>
 int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     static bpdq::SmemOptin optin;
     const int smem = 65536 + MT * kTableBytes;        // tables start at the first 64 KB boundary of the shared window
     if (smem > h->smem_optin)
         return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv: %d bytes of shared memory needed, device offers %d", smem, h->smem_optin);
-    if (const int rc = bpdq::ensure_smem_optin(gemv_lut_kernel<K, MT, D, W, G64>, optin, h->device, smem, "gemv"); rc != BPDQ_OK) return rc;
+    if (const int rc = bpdq::ensure_smem_optin(gemv_lut_kernel<K, MT, D, W, G64, EXT>, optin, h->device, smem, "gemv"); rc != BPDQ_OK) return rc;
     long long total = 0;
     for (int k = 0; k < p.n; ++k) {
         if ((unsigned long long)p.lin[k].blob_bytes >= (1ull << 32))
@@ -605,7 +610,7 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // lets this launch overlap the tail of the kernel before it
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_lut_kernel<K, MT, D, W, G64>, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_lut_kernel<K, MT, D, W, G64, EXT>, p);
     h->launches += 1;
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemv launch: %s", cudaGetErrorString(e));
@@ -616,8 +621,11 @@ int launch_cfg(bpdq_handle_s* h, GemvParams p, cudaStream_t stream) {
 // for every K); one where two tasks do not fit the register file (K = 4).
 template <int K, int MT>
 int launch_one(bpdq_handle_s* h, const GemvParams& p, cudaStream_t stream) {
-    if (p.lin[0].group == 64) return launch_cfg<K, MT, (K <= 3 ? 2 : 1), 16, true>(h, p, stream);
-    return launch_cfg<K, MT, (K <= 3 ? 2 : 1), 16, false>(h, p, stream);
+    bool ext = false;
+    for (int k = 0; k < p.n; ++k) ext = ext || p.lin[k].perm || p.lin[k].bias_a || p.lin[k].conv_b;
+    constexpr int D = K <= 3 ? 2 : 1;
+    if (p.lin[0].group == 64) return ext ? launch_cfg<K, MT, D, 16, true, true>(h, p, stream) : launch_cfg<K, MT, D, 16, true, false>(h, p, stream);
+    return ext ? launch_cfg<K, MT, D, 16, false, true>(h, p, stream) : launch_cfg<K, MT, D, 16, false, false>(h, p, stream);
 }
 
 void fill_linear(GemvLinear& L, const bpdq_handle_s* h) {

@@ -121,7 +121,8 @@ template <int K, bool G64, int NJ> struct Land {
 };
 
 // K planes, MT token tiles of 16, NJ groups of eight rows per task, W warps per CTA
-template <int K, int MT, bool G64, int NJ, int W>
+// EXT: the launch uses a bias or a (gate, up) pair somewhere (kept out of the plain instantiation, which sits at the register cap)
+template <int K, int MT, bool G64, int NJ, int W, bool EXT>
 __global__ void __launch_bounds__(W * 32, 1) gemv_mma_kernel(const __grid_constant__ MmaParams p) {
     using LD = Land<K, G64, NJ>;
     constexpr int NG = LD::kGroups;
@@ -187,7 +188,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_mma_kernel(const __grid_consta
                 const int size = min(L.nrg, (ck + 1) * kChunkRgs) - ck * kChunkRgs;
                 const unsigned mine = (unsigned)((hi - lo) * nsl);
                 const unsigned before = atomicAdd(&L.counters[ck], mine);
-                if (before + mine == (unsigned)(size * L.nslices * L.target_mul)) {
+                if (before + mine == (unsigned)(size * L.nslices * (EXT ? L.target_mul : 1))) {
                     L.counters[ck] = 0u;
                     done[atomicAdd(ndone, 1)] = ck;
                 }
@@ -215,22 +216,24 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_mma_kernel(const __grid_consta
                                 live[u] = true;
                                 row[u] = r;
                                 at[u] = (size_t)(rem / kQuads) * L.out + r;
-                                v[u] = __ldcg(reinterpret_cast<const float4*>(L.conv_a + at[u]));
-                                if (L.conv_b) vb[u] = __ldcg(reinterpret_cast<const float4*>(L.conv_b + at[u]));
+                                v[u] = __ldcg(reinterpret_cast<const float4*>((EXT ? L.conv_a : L.ws) + at[u]));
+                                if (EXT && L.conv_b) vb[u] = __ldcg(reinterpret_cast<const float4*>(L.conv_b + at[u]));
                             }
                         }
                     }
 #pragma unroll
                     for (int u = 0; u < kAhead; ++u) {
                         if (live[u]) {
-                            bpdq::finish_quad(v[u], vb[u], L.bias_a, L.bias_b, L.conv_b != nullptr, row[u]);
-                            if (L.conv_b) __stcg(reinterpret_cast<float4*>(L.conv_b + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
+                            if (EXT) {
+                                bpdq::finish_quad(v[u], vb[u], L.bias_a, L.bias_b, L.conv_b != nullptr, row[u]);
+                                if (L.conv_b) __stcg(reinterpret_cast<float4*>(L.conv_b + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
+                            }
                             const __half2 h01 = __floats2half2_rn(v[u].x, v[u].y), h23 = __floats2half2_rn(v[u].z, v[u].w);
                             uint2 o;
                             o.x = *reinterpret_cast<const unsigned*>(&h01);
                             o.y = *reinterpret_cast<const unsigned*>(&h23);
                             *reinterpret_cast<uint2*>(L.y + at[u]) = o;
-                            __stcg(reinterpret_cast<float4*>(L.conv_a + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
+                            __stcg(reinterpret_cast<float4*>((EXT ? L.conv_a : L.ws) + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
                         }
                     }
                 }
@@ -472,7 +475,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_mma_kernel(const __grid_consta
     if (pend_li >= 0) hand_over(p.lin[pend_li], pend_begin, pend_end, pend_nsl);
 }
 
-template <int K, int MT, bool G64, int NJ, int W>
+template <int K, int MT, bool G64, int NJ, int W, bool EXT>
 int launch_cfg(bpdq_handle_s* h, MmaParams p, cudaStream_t stream) {
     using LD = Land<K, G64, NJ>;
     static bpdq::SmemOptin optin;
@@ -482,7 +485,7 @@ int launch_cfg(bpdq_handle_s* h, MmaParams p, cudaStream_t stream) {
     const int smem = 1024 /*alignment slack*/ + kMiscBytes + MT * ns * kXSliceBytes + W * LD::kBytes;
     if (smem > h->smem_optin)
         return bpdq::set_error(BPDQ_ERR_UNSUPPORTED, "gemv_mma: %d bytes of shared memory needed, device offers %d", smem, h->smem_optin);
-    if (const int rc = bpdq::ensure_smem_optin(gemv_mma_kernel<K, MT, G64, NJ, W>, optin, h->device, smem, "gemv_mma"); rc != BPDQ_OK) return rc;
+    if (const int rc = bpdq::ensure_smem_optin(gemv_mma_kernel<K, MT, G64, NJ, W, EXT>, optin, h->device, smem, "gemv_mma"); rc != BPDQ_OK) return rc;
     p.ns = ns;
     p.dyn_smem = smem;
     long long total = 0;
@@ -517,7 +520,7 @@ int launch_cfg(bpdq_handle_s* h, MmaParams p, cudaStream_t stream) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_mma_kernel<K, MT, G64, NJ, W>, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_mma_kernel<K, MT, G64, NJ, W, EXT>, p);
     h->launches += 1;
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemv_mma launch: %s", cudaGetErrorString(e));
@@ -529,8 +532,14 @@ int launch_cfg(bpdq_handle_s* h, MmaParams p, cudaStream_t stream) {
 template <int K>
 int launch_k(bpdq_handle_s* h, const MmaParams& p, cudaStream_t stream) {
     const bool g64 = p.lin[0].group == 64;
-    if (p.M <= 16) return g64 ? launch_cfg<K, 1, true, 4, 16>(h, p, stream) : launch_cfg<K, 1, false, 4, 16>(h, p, stream);
-    return g64 ? launch_cfg<K, 2, true, 4, 16>(h, p, stream) : launch_cfg<K, 2, false, 4, 16>(h, p, stream);
+    bool ext = false;
+    for (int k = 0; k < p.n; ++k) ext = ext || p.lin[k].bias_a || p.lin[k].conv_b;
+    if (p.M <= 16) {
+        if (ext) return g64 ? launch_cfg<K, 1, true, 4, 16, true>(h, p, stream) : launch_cfg<K, 1, false, 4, 16, true>(h, p, stream);
+        return g64 ? launch_cfg<K, 1, true, 4, 16, false>(h, p, stream) : launch_cfg<K, 1, false, 4, 16, false>(h, p, stream);
+    }
+    if (ext) return g64 ? launch_cfg<K, 2, true, 4, 16, true>(h, p, stream) : launch_cfg<K, 2, false, 4, 16, true>(h, p, stream);
+    return g64 ? launch_cfg<K, 2, true, 4, 16, false>(h, p, stream) : launch_cfg<K, 2, false, 4, 16, false>(h, p, stream);
 }
 
 }  // namespace
