@@ -30,9 +30,10 @@
 // the token columns: tcgen05.ld gives a thread its output row for 16 tokens at a time; adjacent
 // threads hold adjacent output indices, so a warp writes 64 contiguous bytes of y per token.
 //
-// Two kernels share this scheme: gemm_kernel (one output tile per CTA; token tiles of 32..128, two CTAs per SM
-// and a split over the input dimension when tokens are few) and gemm_persistent_kernel (token tile 256: one
-// CTA per SM walks over tiles, two TMEM accumulators, separate epilogue warps; described at its definition).
+// Three kernels share this scheme: gemm_kernel (one output tile per CTA; token tiles of 16..128, two CTAs per SM
+// and a split over the input dimension when tokens are few), gemm_persistent_kernel (129..256 tokens: token tile 256,
+// one CTA per SM walks over tiles, two TMEM accumulators, separate epilogue warps; described at its definition) and
+// gemm_wide_kernel (more than 256 tokens: token tile 512, two issuing warps; bpdq_gemm_wide.cuh).
 //
 // Pipeline of the tile kernel: three rings, each with full / empty mbarriers -- packed blocks (full_p by the
 // copies' bytes, empty_p by one arrival per decode warp once the block is in registers), x tiles (full_b by
@@ -638,9 +639,38 @@ gemm_persistent_kernel(const __grid_constant__ CUtensorMap x_map, const GemmPara
     }
 }
 
+#include "bpdq_gemm_wide.cuh"
+
 // ---- host side ------------------------------------------------------------------------------
 using bpdq::EncodeTiledFn;
 using bpdq::encode_tiled_fn;
+
+// Tensor maps of the blob's planes and coefficients (one box = the K plane segments resp. the coefficient groups of a
+// 128-row x 128-column block), encoded at a handle's first tensor-core launch.
+template <int K>
+int ensure_packed_maps(bpdq_handle_s* h, EncodeTiledFn enc) {
+    if (h->gemm_maps_ready) return BPDQ_OK;
+    const cuuint32_t estr[2] = {1, 1};
+        // planes: rows (block, plane) of out x 16 bytes; coefficients: rows (group, coefficient) of out x 2 bytes; both
+    // as 8-byte elements, so that 128 output rows are 256 resp. 32 elements (a box dimension holds at most 256)
+    const int ng = h->group == 64 ? 2 : 1;
+    const cuuint64_t pd[2] = {(cuuint64_t)h->out * 2, (cuuint64_t)(h->in / 128) * K};
+    const cuuint64_t ps[1] = {(cuuint64_t)h->out * 16};
+    const cuuint32_t pb[2] = {(cuuint32_t)BM * 2, (cuuint32_t)K};
+    const cuuint64_t cd[2] = {(cuuint64_t)h->out / 4, (cuuint64_t)(h->in / h->group) * (K + 1)};
+    const cuuint64_t cs[1] = {(cuuint64_t)h->out * 2};
+    const cuuint32_t cb[2] = {(cuuint32_t)BM / 4, (cuuint32_t)(ng * (K + 1))};
+    CUresult r1 = enc(reinterpret_cast<CUtensorMap*>(h->gemm_maps[0]), CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, h->d_blob, pd, ps, pb, estr,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r2 = enc(reinterpret_cast<CUtensorMap*>(h->gemm_maps[1]), CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, h->d_blob + h->planes_bytes, cd, cs, cb,
+                      estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r1 != CUDA_SUCCESS || r2 != CUDA_SUCCESS)
+        return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: tensor map encode of the packed weights failed (CUresult %d, %d)", (int)r1, (int)r2);
+    h->gemm_maps_ready = 1;
+    return BPDQ_OK;
+}
 
 template <int K, int BN>
 int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
@@ -658,26 +688,7 @@ int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t st
                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (cr != CUDA_SUCCESS) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: tensor map encode failed (CUresult %d)", (int)cr);
-    if (!h->gemm_maps_ready) {
-        // planes: rows (block, plane) of out x 16 bytes; coefficients: rows (group, coefficient) of out x 2 bytes; both
-        // as 8-byte elements, so that 128 output rows are 256 resp. 32 elements (a box dimension holds at most 256)
-        const int ng = h->group == 64 ? 2 : 1;
-        const cuuint64_t pd[2] = {(cuuint64_t)h->out * 2, (cuuint64_t)(h->in / 128) * K};
-        const cuuint64_t ps[1] = {(cuuint64_t)h->out * 16};
-        const cuuint32_t pb[2] = {(cuuint32_t)BM * 2, (cuuint32_t)K};
-        const cuuint64_t cd[2] = {(cuuint64_t)h->out / 4, (cuuint64_t)(h->in / h->group) * (K + 1)};
-        const cuuint64_t cs[1] = {(cuuint64_t)h->out * 2};
-        const cuuint32_t cb[2] = {(cuuint32_t)BM / 4, (cuuint32_t)(ng * (K + 1))};
-        CUresult r1 = enc(reinterpret_cast<CUtensorMap*>(h->gemm_maps[0]), CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, h->d_blob, pd, ps, pb, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        CUresult r2 = enc(reinterpret_cast<CUtensorMap*>(h->gemm_maps[1]), CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, h->d_blob + h->planes_bytes, cd, cs, cb,
-                          estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r1 != CUDA_SUCCESS || r2 != CUDA_SUCCESS)
-            return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: tensor map encode of the packed weights failed (CUresult %d, %d)", (int)r1, (int)r2);
-        h->gemm_maps_ready = 1;
-    }
+    if (const int rc = ensure_packed_maps<K>(h, enc); rc != BPDQ_OK) return rc;
     GemmParams p;
     p.blob = h->d_blob; p.planes_bytes = h->planes_bytes; p.y = static_cast<__half*>(y); p.status = h->d_status;
     p.out = h->out; p.in = h->in; p.group = h->group; p.M = M;
@@ -734,12 +745,44 @@ int launch_persistent(bpdq_handle_s* h, const void* x, void* y, int M, cudaStrea
 }
 
 template <int K>
+int launch_wide(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
+    using C = WideCfg<K>;
+    static bpdq::SmemOptin optin;
+    if (const int rc = bpdq::ensure_smem_optin(gemm_wide_kernel<K>, optin, h->device, C::kSmemBytes, "gemm"); rc != BPDQ_OK) return rc;
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: cuTensorMapEncodeTiled is not available from this driver");
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)h->in, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)h->in * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kWideBK, 256};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult cr = enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm: tensor map encode failed (CUresult %d)", (int)cr);
+    if (const int rc = ensure_packed_maps<K>(h, enc); rc != BPDQ_OK) return rc;
+    GemmParams p;
+    p.blob = h->d_blob; p.planes_bytes = h->planes_bytes; p.y = static_cast<__half*>(y); p.status = h->d_status;
+    p.out = h->out; p.in = h->in; p.group = h->group; p.M = M;
+    p.ws = h->d_ws; p.counters = h->d_counters; p.kb_per = h->in / kWideBK; p.bias = static_cast<const __half*>(h->d_bias);
+    const long long ntiles = (long long)((h->out + BM - 1) / BM) * ((M + kWideBN - 1) / kWideBN);
+    const int grid = ntiles < h->sm_count ? (int)ntiles : h->sm_count;
+    gemm_wide_kernel<K><<<grid, kWideThreads, C::kSmemBytes, stream>>>(map, *reinterpret_cast<const CUtensorMap*>(h->gemm_maps[0]),
+                                                                      *reinterpret_cast<const CUtensorMap*>(h->gemm_maps[1]), p);
+    h->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return bpdq::set_error(BPDQ_ERR_CUDA, "gemm launch: %s", cudaGetErrorString(e));
+    return BPDQ_OK;
+}
+
+template <int K>
 int launch_k(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream) {
     if (M <= 16) return launch_tile<K, 16>(h, x, y, M, stream);
     if (M <= 32) return launch_tile<K, 32>(h, x, y, M, stream);
     if (M <= 64) return launch_tile<K, 64>(h, x, y, M, stream);
     if (M <= 128) return launch_tile<K, 128>(h, x, y, M, stream);
-    return launch_persistent<K>(h, x, y, M, stream);
+    if (M <= 256) return launch_persistent<K>(h, x, y, M, stream);
+    return launch_wide<K>(h, x, y, M, stream);       // 512-token tiles: measured faster than the 256-token kernel from 257 tokens on
 }
 
 }  // namespace

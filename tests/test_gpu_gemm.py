@@ -30,6 +30,12 @@ pytestmark = pytest.mark.gpu
     (3, 64, 160, 640, 24),       # tile kernel, ragged last row tile (the tensor maps fill the missing rows), two groups per block
     (1, 256, 144, 1024, 100),    # tile kernel with the 128-token tile, ragged row tile, a group every two blocks
     (2, 128, 400, 1152, 9),      # 16-token tile, odd number of blocks, rings wrap at different stages
+    (2, 128, 256, 512, 256),     # the most tokens the 256-token kernel takes
+    (3, 128, 384, 2048, 200),    # 256-token kernel, ragged token tile
+    (2, 64, 160, 640, 700),      # 512-token kernel: two token tiles (the second holds 188), ragged row tile, a group per half block
+    (3, 256, 272, 1024, 513),    # 512-token kernel: the second token tile holds one token; a group every two blocks
+    (1, 128, 128, 256, 1030),    # 512-token kernel: two blocks per tile, three token tiles
+    (4, 128, 256, 384, 300),     # 512-token kernel with sixteen candidates (largest packed blocks), odd number of blocks per tile
 ])
 def test_gemm_kernel(K, g, out, in_, M):
     h, bits, coef = G.make_layer(60 + K, out, in_, K, g, max_M=M)
