@@ -45,9 +45,9 @@ FALLBACK_HBM_GBS, FALLBACK_TFLOPS = 6650.0, 1590.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the headline launch, from the ncu capture summarised in
 # profiles/gemv_lut_K2_layer72b_batch_M1.md (set to None whenever the kernel changes until the counters are taken again)
 GEMV_TRAFFIC_BYTES_PER_LAUNCH = 264_366_080
-# the same for one launch of the persistent tcgen05 kernel on the gate projection at K = 3, M = 2048
-# (profiles/gemm_K3_gate_29568x8192_M2048.md); the prefill sections time whole layers, so this is context for them
-GEMM_GATE_K3_M2048_TRAFFIC_BYTES = None
+# the same for one launch of the 512-token tcgen05 kernel on the gate projection at K = 3, M = 2048
+# (profiles/gemm_wide_K3_gate_29568x8192_M2048.md); the prefill sections time whole layers, so this is context for them
+GEMM_GATE_K3_M2048_TRAFFIC_BYTES = 553_668_096
 TIMED_BLOCKS = 25
 
 
@@ -586,7 +586,7 @@ def extra_sections(torch, binding, args, peaks, sp, stream):
         tf = flops / (ms * 1e-3) / 1e12
         out[f"prefill_gemm_layer_K{K}_M{M}"] = {
             "ms_per_layer": ms, "tflops": tf, "per_linear": per,
-            "roofline": {"bound": "tensor", "kernel": "gemm_persistent_kernel", "achieved": tf, "peak": peaks["tflops"], "unit": "TFLOP/s",
+            "roofline": {"bound": "tensor", "kernel": "gemm_wide_kernel", "achieved": tf, "peak": peaks["tflops"], "unit": "TFLOP/s",
                          "frac": tf / peaks["tflops"], "frac_of_sustained": tf / peaks["tflops_sustained"],
                          "peak_source": peaks["source"] + " bf16 burst (fp16 has the same nominal rate)",
                          "traffic": None, "traffic_gate_launch_K3_M2048": GEMM_GATE_K3_M2048_TRAFFIC_BYTES}}
