@@ -258,6 +258,12 @@ BPDQ_API int bpdq_read_blob(bpdq_handle_t h, void* host_blob);
  * then undefined; the context stays usable).  Clears the word. */
 BPDQ_API int bpdq_get_status(bpdq_handle_t h, void* stream);
 
+/* Diagnostic for the bounded device-side waits: enqueues a one-warp kernel that waits, with the bounded wait every
+ * kernel of the library uses (cut to 50 ms; the kernels allow two seconds), on a barrier that nothing arrives at.  The wait gives up,
+ * records BPDQ_ERR_TIMEOUT in the handle's status word and the kernel ends normally: the next bpdq_get_status
+ * returns BPDQ_ERR_TIMEOUT once and the handle stays usable.  Nothing else is touched. */
+BPDQ_API int bpdq_probe_wait_limit(bpdq_handle_t h, void* stream);
+
 /* Number of kernels this handle has launched since creation (bookkeeping for benchmarks). */
 BPDQ_API int bpdq_launch_count(bpdq_handle_t h, uint64_t* count);
 

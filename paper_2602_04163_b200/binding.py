@@ -23,7 +23,7 @@ NOALLOC_MAX_OUT = 65536
 
 EXPORTS = ("bpdq_packed_bytes", "bpdq_pack", "bpdq_unpack", "bpdq_create", "bpdq_dequant", "bpdq_linear",
            "bpdq_linear_ex", "bpdq_linear_host", "bpdq_set_gemv_max_m", "bpdq_set_few_max_m", "bpdq_read_blob", "bpdq_get_status",
-           "bpdq_launch_count", "bpdq_destroy", "bpdq_quantize_datafree", "bpdq_truncate_planes", "bpdq_set_input_permutation", "bpdq_set_bias", "bpdq_gate_up_swiglu", "bpdq_last_error", "bpdq_linear_noalloc", "bpdq_linear_batch", "bpdq_linear_batch_host")
+           "bpdq_launch_count", "bpdq_destroy", "bpdq_quantize_datafree", "bpdq_truncate_planes", "bpdq_set_input_permutation", "bpdq_set_bias", "bpdq_gate_up_swiglu", "bpdq_probe_wait_limit", "bpdq_last_error", "bpdq_linear_noalloc", "bpdq_linear_batch", "bpdq_linear_batch_host")
 
 _lib = None
 
@@ -64,6 +64,7 @@ def lib() -> ctypes.CDLL:
         L.bpdq_gate_up_swiglu.argtypes = [vp, vp, vp, vp, i, vp]
         L.bpdq_read_blob.argtypes = [vp, vp]
         L.bpdq_get_status.argtypes = [vp, vp]
+        L.bpdq_probe_wait_limit.argtypes = [vp, vp]
         L.bpdq_launch_count.argtypes = [vp, ctypes.POINTER(u64)]
         L.bpdq_destroy.argtypes = [vp]
         L.bpdq_last_error.argtypes = []
@@ -229,6 +230,9 @@ class Handle:
 
     def bpdq_get_status(self, stream: int = 0) -> None:
         _check(lib().bpdq_get_status(self._h, stream))
+
+    def bpdq_probe_wait_limit(self, stream: int = 0) -> None:
+        _check(lib().bpdq_probe_wait_limit(self._h, stream))
 
     def bpdq_launch_count(self) -> int:
         c = ctypes.c_uint64()

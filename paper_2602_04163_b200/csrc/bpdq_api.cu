@@ -158,8 +158,8 @@ extern "C" int bpdq_create(bpdq_handle_t* hp, int out, int in, int K, int group,
     // Measured on 72B-shaped layers: one two-token pass of the look-up-table kernel (37 us on the largest projections)
     // beats every other kernel; a second pass (64 us) does not beat the few-token kernel.
     h->gemv_max_m = 2;
-    // 3 to 16 tokens: the few-token kernel reads the weights once (45-60 us on the largest 72B-shaped projections
-    // against 64 us for two look-up-table passes and 67-75 us for the tcgen05 tile kernel); from 17 tokens on its second
+    // 3 to 16 tokens: the few-token kernel reads the weights once (43-60 us on the largest 72B-shaped projections
+    // against 64 us for two look-up-table passes and 67-78 us for the tcgen05 tile kernel); from 17 tokens on its second
     // token tile costs more than the tile kernel.
     h->few_max_m = 16;
     if (K == 4) { h->gemv_max_m = 4; h->few_max_m = 0; }   // sixteen candidates: the few-token kernel's decode no longer fits its registers (110 us), two look-up-table passes do better
@@ -400,6 +400,12 @@ extern "C" int bpdq_get_status(bpdq_handle_t h, void* stream) {
     if (e != cudaSuccess) return cuda_fail("bpdq_get_status", e);
     if (st != BPDQ_OK) return set_error(st, "a device-side bounded wait expired (status %d)", st);
     return BPDQ_OK;
+}
+
+extern "C" int bpdq_probe_wait_limit(bpdq_handle_t h, void* stream) {
+    if (!h) return set_error(BPDQ_ERR_INVALID, "bpdq_probe_wait_limit: null handle");
+    if (const int rc = check_device(h, "bpdq_probe_wait_limit"); rc != BPDQ_OK) return rc;
+    return launch_wait_limit_probe(h, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int bpdq_launch_count(bpdq_handle_t h, uint64_t* count) {

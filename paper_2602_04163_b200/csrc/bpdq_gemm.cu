@@ -139,10 +139,7 @@ __host__ __device__ constexpr unsigned instr_desc_f16(int m, int n) {
 // Ring depths of the tile kernel.  Its three operand streams have very different sizes per 64-column stage -- 16 KB of
 // decoded weights (A), BN x 128 bytes of activations (B), about 2.5 KB of packed planes and coefficients -- and very
 // different latencies (A is produced on the SM, B comes from L2, the packed bytes from HBM), so each has its own
-// ring: a few A slots, more B slots, and packed 128-column blocks several stages ahead.  A 72B-shaped projection at
-// M <= 64 takes 80 us this way (88 us with one common ring of three or four stages and bulk copies per segment); what
-// remains is hand-over latency: the decode warps and the single MMA thread each wait for the other about half of the
-// time (cycle counters in a working copy), whatever the ring depths.
+// ring: a few A slots, more B slots, and packed 128-column blocks several stages ahead.
 template <int K, int BN> struct TileCfg {
     static constexpr int kBTileBytes = BN * BK * 2;
     static constexpr int kPlaneBytes = K * BM * 16;             // K segments of 128 rows x 16 bytes
@@ -228,6 +225,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
             // ragged last tile are filled with zeros (and count as received bytes).
             int pb = 0, xb = 0;                          // next packed block, next x stage
             unsigned idle = 0;
+            unsigned long long idle_since = 0;
             while (pb < nblk || xb < nst) {
                 bool moved = false;
                 if (pb < nblk && mbar_try_wait(empty_p(pb % SP), ((unsigned)(pb / SP) & 1u) ^ 1u)) {
@@ -248,12 +246,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
                 }
                 if (moved) {
                     idle = 0;
-                } else if (++idle >= kWaitLimit) {       // neither ring has freed a slot for too long
-                    *abort_flag = 1;
-                    atomicExch(p.status, BPDQ_ERR_TIMEOUT);
-                    break;
-                } else if ((idle & 63u) == 63u && *abort_flag) {
-                    break;
+                } else if (++idle == 1) {
+                    idle_since = global_ns();
+                } else if ((idle & 63u) == 63u) {
+                    if (*abort_flag) break;
+                    if (global_ns() - idle_since > kWaitNanos) {   // neither ring has freed a slot for too long
+                        *abort_flag = 1;
+                        atomicExch(p.status, BPDQ_ERR_TIMEOUT);
+                        break;
+                    }
                 }
             }
         }
@@ -785,9 +786,32 @@ int launch_k(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t strea
     return launch_wide<K>(h, x, y, M, stream);       // 512-token tiles: measured faster than the 256-token kernel from 257 tokens on
 }
 
+// Diagnostic: the library's bounded wait on a barrier that nothing arrives at.  It must give up after its limit, record
+// BPDQ_ERR_TIMEOUT in the status word and let the kernel end normally.
+__global__ void wait_limit_probe_kernel(int* status) {
+    __shared__ alignas(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_wait_ns(smem_u32(&bar), 0u, &abort_flag, status, 50000000ull);   // 50 ms here; the kernels allow two seconds
+    __syncthreads();
+}
+
 }  // namespace
 
 namespace bpdq {
+
+int launch_wait_limit_probe(bpdq_handle_s* h, cudaStream_t stream) {
+    wait_limit_probe_kernel<<<1, 32, 0, stream>>>(h->d_status);
+    h->launches += 1;
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return set_error(BPDQ_ERR_CUDA, "probe launch: %s", cudaGetErrorString(e));
+    return BPDQ_OK;
+}
 
 EncodeTiledFn encode_tiled_fn() {
     static EncodeTiledFn fn = nullptr;

@@ -97,6 +97,7 @@ int launch_gemv_simple(bpdq_handle_s* h, const void* x, void* y, int M, cudaStre
 int launch_gemv(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
 int launch_gemv_batch(bpdq_handle_s* const* hs, const void* const* xs, void* const* ys, int n, int M, cudaStream_t stream, bool pair = false);
 int launch_gemm(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);
+int launch_wait_limit_probe(bpdq_handle_s* h, cudaStream_t stream);
 int launch_gather_columns(bpdq_handle_s* h, const void* x, int M, cudaStream_t stream);   // x[m][perm[j]] -> d_xperm[m][j]
 int launch_swiglu(const void* gate, const void* up, void* hout, size_t n, cudaStream_t stream);
 int launch_gemv_mma(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t stream);

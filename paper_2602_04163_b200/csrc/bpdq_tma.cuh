@@ -16,8 +16,6 @@ EncodeTiledFn encode_tiled_fn();      // null when the driver does not offer cuT
 #if defined(__CUDACC__)
 namespace tma {
 
-constexpr unsigned kWaitLimit = 1u << 24;                      // polls of try_wait before a wait gives up
-
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
@@ -38,15 +36,31 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false if the CTA has been aborted or the limit ran out (and aborts it).
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag, int* status) {
-    for (unsigned n = 0; n < kWaitLimit; ++n) {
+// Bounded wait: gives up after max_ns nanoseconds (mbarrier.try_wait itself blocks for a hardware-defined slice per
+// poll, so the bound is taken on the clock, read every 64 polls, not on the poll count).  Returns false if the CTA has
+// been aborted or the limit ran out (and aborts it, recording BPDQ_ERR_TIMEOUT in the status word).
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ bool mbar_wait_ns(unsigned bar, unsigned parity, volatile int* abort_flag, int* status, unsigned long long max_ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (unsigned n = 1;; ++n) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((n & 63u) == 63u && *abort_flag) return false;
+        if ((n & 63u) == 63u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > max_ns) break;
+        }
     }
     *abort_flag = 1;
     atomicExch(status, BPDQ_ERR_TIMEOUT);
     return false;
+}
+constexpr unsigned long long kWaitNanos = 2000000000ull;       // two seconds: far beyond any wait of a healthy launch
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag, int* status) {
+    return mbar_wait_ns(bar, parity, abort_flag, status, kWaitNanos);
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }

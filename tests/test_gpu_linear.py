@@ -133,3 +133,18 @@ def test_chain_of_dependent_launches(M):
         G.assert_linear_close(y.cpu().numpy().astype(np.float64), y_ref, a_ref, f"stage {k}")
         src = y
     assert not torch.equal(inputs[0], inputs[1])
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_handle_usable():
+    """Every device-side wait of the library is bounded.  A barrier that nothing arrives at makes one run out: the status
+    word then says BPDQ_ERR_TIMEOUT (once), the kernel ends by itself, and the same handle computes correctly afterwards."""
+    h, bits, coef = G.make_layer(601, 160, 640, 2, 128, max_M=40)
+    sp = G.stream_ptr()
+    h.bpdq_get_status(sp)                                                # clean to begin with
+    h.bpdq_probe_wait_limit(sp)
+    with pytest.raises(binding.BpdqError) as ei:
+        h.bpdq_get_status(sp)
+    assert ei.value.code == binding.ERR_TIMEOUT
+    h.bpdq_get_status(sp)                                                # reading the word cleared it
+    for M, kernel in ((1, binding.KERNEL_GEMV), (5, binding.KERNEL_FEW), (40, binding.KERNEL_GEMM)):
+        G.check_linear(h, bits, coef, synth.activations(602 + M, M, 640), 128, kernel, what=f"after the probe M={M}")
