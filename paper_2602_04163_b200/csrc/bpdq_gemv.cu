@@ -120,6 +120,10 @@ __device__ __forceinline__ unsigned short ldg_stream2(const uint8_t* p) {
     asm volatile("ld.global.nc.L1::no_allocate.u16 %0, [%1];" : "=h"(v) : "l"(p));
     return v;
 }
+// add into the workspace without a returned value: nothing for the warp to wait on
+__device__ __forceinline__ void red_add(float* p, float v) {
+    asm volatile("red.global.add.f32 [%0], %1;" :: "l"(p), "f"(v) : "memory");
+}
 // Table load.  Not volatile: its address is computed from plane bytes that were read after the
 // barrier that published the tables, so it cannot move above that barrier, and the compiler may
 // interleave the independent look-ups of a plane unit freely.
@@ -221,6 +225,55 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
     const int t_end = p.t_begin[bid + 1];
     int li = 0;                                       // linear that task t belongs to
 
+    // rows of the chunks on the completion list: rounded to binary16, written to y, workspace zeroed again
+    auto convert_done = [&](const GemvLinear& L) {
+        const int nd = *ndone;
+        if (nd > 0) {
+            __threadfence();
+            // items of four consecutive rows; a thread reads several before it writes, so that the
+            // L2 round trips of a CTA that completes many chunks overlap
+            constexpr int kQuads = kChunkRgs * 16 / 4, kAhead = 4;
+            const int nitems = nd * MT * kQuads;
+            for (int i0 = tid; i0 < nitems; i0 += kThreads * kAhead) {
+                float4 v[kAhead], vb[kAhead];
+                size_t at[kAhead];
+                int row[kAhead];
+                bool live[kAhead];
+#pragma unroll
+                for (int u = 0; u < kAhead; ++u) {
+                    const int idx = i0 + u * kThreads;
+                    live[u] = false;
+                    if (idx < nitems) {
+                        const int ckd = done[idx / (MT * kQuads)];
+                        const int rem = idx % (MT * kQuads);
+                        const int r = ckd * kChunkRgs * 16 + (rem % kQuads) * 4;
+                        if (r < L.out) {                  // out is a multiple of 16: a quad is inside or outside as a whole
+                            live[u] = true;
+                            row[u] = r;
+                            at[u] = (size_t)(rem / kQuads) * L.out + r;
+                            v[u] = __ldcg(reinterpret_cast<const float4*>((EXT ? L.conv_a : L.ws) + at[u]));
+                            if (EXT && L.conv_b) vb[u] = __ldcg(reinterpret_cast<const float4*>(L.conv_b + at[u]));
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kAhead; ++u) {
+                    if (live[u]) {
+                        if (EXT) {
+                            bpdq::finish_quad(v[u], vb[u], L.bias_a, L.bias_b, L.conv_b != nullptr, row[u]);
+                            if (L.conv_b) __stcg(reinterpret_cast<float4*>(L.conv_b + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
+                        }
+                        const __half2 h01 = __floats2half2_rn(v[u].x, v[u].y), h23 = __floats2half2_rn(v[u].z, v[u].w);
+                        uint2 o;
+                        o.x = *reinterpret_cast<const unsigned*>(&h01);
+                        o.y = *reinterpret_cast<const unsigned*>(&h23);
+                        *reinterpret_cast<uint2*>(L.y + at[u]) = o;
+                        __stcg(reinterpret_cast<float4*>((EXT ? L.conv_a : L.ws) + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
+                    }
+                }
+            }
+        }
+    };
     // ---- hand-over of a finished segment ----
     // Row sums are accumulated across slices with binary32 atomic adds in `ws` (kept zero
     // between calls).  Row groups are counted in chunks of kChunkRgs; whoever delivers the last
@@ -241,52 +294,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                 }
             }
             __syncthreads();
-            const int nd = *ndone;
-            if (nd > 0) {
-                __threadfence();
-                // items of four consecutive rows; a thread reads several before it writes, so that the
-                // L2 round trips of a CTA that completes many chunks overlap
-                constexpr int kQuads = kChunkRgs * 16 / 4, kAhead = 4;
-                const int nitems = nd * MT * kQuads;
-                for (int i0 = tid; i0 < nitems; i0 += kThreads * kAhead) {
-                    float4 v[kAhead], vb[kAhead];
-                    size_t at[kAhead];
-                    int row[kAhead];
-                    bool live[kAhead];
-#pragma unroll
-                    for (int u = 0; u < kAhead; ++u) {
-                        const int idx = i0 + u * kThreads;
-                        live[u] = false;
-                        if (idx < nitems) {
-                            const int ckd = done[idx / (MT * kQuads)];
-                            const int rem = idx % (MT * kQuads);
-                            const int r = ckd * kChunkRgs * 16 + (rem % kQuads) * 4;
-                            if (r < L.out) {                  // out is a multiple of 16: a quad is inside or outside as a whole
-                                live[u] = true;
-                                row[u] = r;
-                                at[u] = (size_t)(rem / kQuads) * L.out + r;
-                                v[u] = __ldcg(reinterpret_cast<const float4*>((EXT ? L.conv_a : L.ws) + at[u]));
-                                if (EXT && L.conv_b) vb[u] = __ldcg(reinterpret_cast<const float4*>(L.conv_b + at[u]));
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < kAhead; ++u) {
-                        if (live[u]) {
-                            if (EXT) {
-                                bpdq::finish_quad(v[u], vb[u], L.bias_a, L.bias_b, L.conv_b != nullptr, row[u]);
-                                if (L.conv_b) __stcg(reinterpret_cast<float4*>(L.conv_b + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
-                            }
-                            const __half2 h01 = __floats2half2_rn(v[u].x, v[u].y), h23 = __floats2half2_rn(v[u].z, v[u].w);
-                            uint2 o;
-                            o.x = *reinterpret_cast<const unsigned*>(&h01);
-                            o.y = *reinterpret_cast<const unsigned*>(&h23);
-                            *reinterpret_cast<uint2*>(L.y + at[u]) = o;
-                            __stcg(reinterpret_cast<float4*>((EXT ? L.conv_a : L.ws) + at[u]), make_float4(0.f, 0.f, 0.f, 0.f));
-                        }
-                    }
-                }
-            }
+            convert_done(L);
             __syncthreads();
         }
     };
@@ -320,31 +328,33 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                 csrc[q] = (unsigned)L.planes_bytes + ((unsigned)G * (K + 1) * L.out + r) * 2u;
             }
         }
-        auto load_task = [&](Task<K, NG>& tk, int n) {
+        // one half of a task: the plane units and coefficients of the lane's block in block pair q
+        auto load_half = [&](Task<K, NG>& tk, int n, int q) {
+            if (valid[q]) {
+                const unsigned ps = psrc[q] + (unsigned)n * (W * 256);
 #pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                if (valid[q]) {
-                    const unsigned ps = psrc[q] + (unsigned)n * (W * 256);
+                for (int i = 0; i < K; ++i) tk.pl[q][i] = ldg_stream16(L.blob + (size_t)(ps + i * plane_pitch));
+                const unsigned cs = csrc[q] + (unsigned)n * (W * 32);
+                if constexpr (NG == 2) {          // the pair's even row, group a & 1 (rows are even-aligned: out is a multiple of 16)
+                    const unsigned cp = cs - 2u * (a & 1) + (unsigned)(a & 1) * (K + 1) * coef_pitch;
 #pragma unroll
-                    for (int i = 0; i < K; ++i) tk.pl[q][i] = ldg_stream16(L.blob + (size_t)(ps + i * plane_pitch));
-                    const unsigned cs = csrc[q] + (unsigned)n * (W * 32);
-                    if constexpr (NG == 2) {          // the pair's even row, group a & 1 (rows are even-aligned: out is a multiple of 16)
-                        const unsigned cp = cs - 2u * (a & 1) + (unsigned)(a & 1) * (K + 1) * coef_pitch;
+                    for (int i = 0; i <= K; ++i) tk.cfp[q][i] = ldg_stream4(L.blob + (size_t)(cp + i * coef_pitch));
+                } else {
 #pragma unroll
-                        for (int i = 0; i <= K; ++i) tk.cfp[q][i] = ldg_stream4(L.blob + (size_t)(cp + i * coef_pitch));
-                    } else {
+                    for (int i = 0; i <= K; ++i) tk.cf[q][i] = ldg_stream2(L.blob + (size_t)(cs + i * coef_pitch));
+                }
+            } else {                              // contributes nothing: zero planes, zero coefficients
 #pragma unroll
-                        for (int i = 0; i <= K; ++i) tk.cf[q][i] = ldg_stream2(L.blob + (size_t)(cs + i * coef_pitch));
-                    }
-                } else {                              // contributes nothing: zero planes, zero coefficients
+                for (int i = 0; i < K; ++i) tk.pl[q][i] = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                    for (int i = 0; i < K; ++i) tk.pl[q][i] = make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-                    for (int i = 0; i <= K; ++i) {
-                        if constexpr (NG == 2) tk.cfp[q][i] = 0u; else tk.cf[q][i] = 0;
-                    }
+                for (int i = 0; i <= K; ++i) {
+                    if constexpr (NG == 2) tk.cfp[q][i] = 0u; else tk.cf[q][i] = 0;
                 }
             }
+        };
+        auto load_task = [&](Task<K, NG>& tk, int n) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) load_half(tk, n, q);
         };
 
         // ---- this thread's inputs for the table build and the first tasks' weights ----
@@ -424,7 +434,11 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
         __syncthreads();
 
         // ---- stream the row groups of this slice ----
-        auto process_task = [&](const Task<K, NG>& tk, int n) {
+        // n_next >= 0: the task that takes this one's registers; each half is requested as soon as the half it
+        // replaces has been used, so that nearly D tasks per warp are in flight rather than D - 1 (three planes
+        // for two tokens keep the whole-task request: the other order costs that instantiation spills)
+        constexpr bool kReloadHalves = !(K == 3 && MT == 2);
+        auto process_task = [&](Task<K, NG>& tk, int n, int n_next) {
             float yacc[MT];
 #pragma unroll
             for (int m = 0; m < MT; ++m) yacc[m] = 0.f;
@@ -537,6 +551,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                         for (int m = 0; m < MT; ++m) yacc[m] = fmaf(ci, S[i * MT + m], yacc[m]);
                     }
                 }
+                if (kReloadHalves && n_next >= 0) load_half(tk, n_next, q);
             }
             // the two half-warps hold the even-block and odd-block parts of the same 16 rows
 #pragma unroll
@@ -544,7 +559,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
             if (h == 0) {
                 const int r = (rg_begin + wid + n * W) * 16 + a;
 #pragma unroll
-                for (int m = 0; m < MT; ++m) atomicAdd(&L.ws[(size_t)m * L.out + r], yacc[m]);
+                for (int m = 0; m < MT; ++m) red_add(&L.ws[(size_t)m * L.out + r], yacc[m]);
             }
         };
         for (int n0 = 0; n0 < ntask; n0 += D) {
@@ -552,8 +567,12 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
             for (int d = 0; d < D; ++d) {
                 const int n = n0 + d;
                 if (n < ntask) {                      // warp-uniform
-                    process_task(tk[d], n);
-                    if (n + D < ntask) load_task(tk[d], n + D);
+                    if constexpr (kReloadHalves) {
+                        process_task(tk[d], n, n + D < ntask ? n + D : -1);
+                    } else {
+                        process_task(tk[d], n, -1);
+                        if (n + D < ntask) load_task(tk[d], n + D);
+                    }
                 }
             }
         }
