@@ -44,7 +44,7 @@ HBM_NOMINAL_GBS = 8000.0
 FALLBACK_HBM_GBS, FALLBACK_TFLOPS = 6650.0, 1590.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the headline launch, from the ncu capture summarised in
 # profiles/gemv_lut_K2_layer72b_batch_M1.md (set to None whenever the kernel changes until the counters are taken again)
-GEMV_TRAFFIC_BYTES_PER_LAUNCH = 264_366_080
+GEMV_TRAFFIC_BYTES_PER_LAUNCH = 264_899_840
 # the same for one launch of the 512-token tcgen05 kernel on the gate projection at K = 3, M = 2048
 # (profiles/gemm_wide_K3_gate_29568x8192_M2048.md); the prefill sections time whole layers, so this is context for them
 GEMM_GATE_K3_M2048_TRAFFIC_BYTES = 553_668_096
