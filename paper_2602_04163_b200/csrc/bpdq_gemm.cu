@@ -145,8 +145,8 @@ template <int K, int BN> struct TileCfg {
     static constexpr int kPlaneBytes = K * BM * 16;             // K segments of 128 rows x 16 bytes
     static constexpr int kCoefBytes = (K + 1) * BM * 2;         // K+1 segments of 128 rows x 2 bytes: one coefficient group
     static constexpr int kBlockBytes = (kPlaneBytes + 2 * kCoefBytes + 1023) / 1024 * 1024;   // a block's planes and up to two groups (g = 64)
-    static constexpr int kCtasPerSm = BN <= 64 ? 2 : 1;         // few tokens: bound by the decode threads, so two CTAs share an SM
-    static constexpr int kSmemBudget = kCtasPerSm == 2 ? 111 * 1024 : 222 * 1024;
+    static constexpr int kCtasPerSm = 2;                        // bound by the decode threads, so two CTAs share an SM (128 tokens: with two x slots)
+    static constexpr int kSmemBudget = 111 * 1024;
     // One thread issues a tcgen05.mma every 160 clocks or so whatever its shape, while the pipe could take one of these
     // few-column MMAs every 40 to 50 clocks: up to 32 tokens two warps issue, stage `it` going to issuer it % 2, each into
     // an accumulator of its own (added up in the epilogue).  A parity wait is only safe on consecutive phases, so every
@@ -156,8 +156,8 @@ template <int K, int BN> struct TileCfg {
     // use u of a slot (stage it) has, for the stage it stored before (it - 1 or it - 3), already waited for an MMA no
     // earlier than it - 6, the one that ended use u - 2; MMAs complete in order, so the wait is on the next phase.
     static constexpr int kIssuers = BN <= 32 ? 2 : 1;
-    static constexpr int kSA = kIssuers == 2 ? 4 : (BN <= 64 ? 3 : 4);
-    static constexpr int kSB = BN <= 16 ? 8 : (BN <= 32 ? (K <= 3 ? 6 : 4) : 4);
+    static constexpr int kSA = kIssuers == 2 ? 4 : 3;
+    static constexpr int kSB = BN <= 16 ? 8 : (BN <= 32 ? (K <= 3 ? 6 : 4) : (BN <= 64 ? 4 : 2));
     static constexpr int kRest = kSmemBudget - kSA * kATileBytes - kSB * kBTileBytes - 2048;
     static constexpr int kSP = (kRest / kBlockBytes > 8 ? 8 : kRest / kBlockBytes) / kDecodeGroups * kDecodeGroups;
     static_assert(kSP >= 2, "at least two packed blocks in flight");
@@ -701,7 +701,8 @@ int launch_tile(bpdq_handle_s* h, const void* x, void* y, int M, cudaStream_t st
         // fewer output tiles than CTA slots: split the input dimension so that every SM gets work
         const int slots = h->sm_count * C::kCtasPerSm;
         int splits = slots / (int)grid.x;
-        if (splits > 8) splits = 8;
+        constexpr int kMaxSplits = BN <= 32 ? 8 : 4;   // every split adds BN x 128 atomic adds per tile: fewer with many tokens
+        if (splits > kMaxSplits) splits = kMaxSplits;
         if (splits > nkb / 16) splits = nkb / 16;     // at least 16 stages (1024 columns) per CTA
         if (splits > 1) {
             p.kb_per = ((nkb + splits - 1) / splits + 1) / 2 * 2;

@@ -695,7 +695,7 @@ bool gemv_supported(int out, int in, int K, int group) {
 // binary32 row sums: kMaxMT tokens for the look-up-table kernel; up to 64 tokens for the tensor-core kernel's split
 // over the input dimension
 size_t gemv_workspace_bytes(int out, int, int, int, int max_M, int) {
-    const int tokens = max_M < kMaxMT ? kMaxMT : (max_M > 64 ? 64 : max_M);
+    const int tokens = max_M < kMaxMT ? kMaxMT : (max_M > 128 ? 128 : max_M);   // the tile kernel's split over the input dimension shares it, up to its largest token tile
     return (size_t)tokens * out * sizeof(float);
 }
 

@@ -25,6 +25,8 @@ pytestmark = pytest.mark.gpu
     (2, 128, 256, 4096, 40),     # few row tiles, long rows: four CTAs share an output tile (split over the input dimension)
     (3, 64, 128, 8192, 64),      # eight-way split
     (4, 128, 384, 2048, 7),      # two-way split, ragged token tile
+    (2, 128, 256, 4096, 100),    # 128-token tile shared by four CTAs (split over the input dimension), two CTAs per SM
+    (3, 128, 384, 2048, 128),    # 128-token tile, two-way split, all 128 token columns in use
     (2, 128, 256, 384, 20500),   # 162 output tiles for 148 persistent CTAs: a second tile per CTA, odd number of blocks per tile
     (4, 128, 128, 640, 38000),   # 149 tiles, three-stage ring (K = 4), odd number of blocks per tile
     (3, 64, 160, 640, 24),       # tile kernel, ragged last row tile (the tensor maps fill the missing rows), two groups per block
@@ -46,7 +48,7 @@ def test_gemm_kernel(K, g, out, in_, M):
     G.check_linear(h, bits, coef, x, g, binding.KERNEL_GEMM, rows=rows, what="gemm")
     y1 = G.run_linear(h, x, binding.KERNEL_GEMM)
     y2 = G.run_linear(h, x, binding.KERNEL_GEMM)
-    if M > 64 or in_ < 2048:
+    if M > 128 or in_ < 2048:
         assert np.array_equal(y1, y2)                    # one CTA per output tile, fixed accumulation order: bit-identical reruns
     else:                                                # CTAs that share a tile add their parts in a free order: last binary16 digit
         assert np.allclose(y1, y2, rtol=2.0 ** -9, atol=1e-5)
