@@ -148,16 +148,16 @@ template <int K, int BN> struct TileCfg {
     static constexpr int kCtasPerSm = 2;                        // bound by the decode threads, so two CTAs share an SM (128 tokens: with two x slots)
     static constexpr int kSmemBudget = 111 * 1024;
     // One thread issues a tcgen05.mma every 160 clocks or so whatever its shape, while the pipe could take one of these
-    // few-column MMAs every 40 to 50 clocks: up to 32 tokens two warps issue, stage `it` going to issuer it % 2, each into
+    // few-column MMAs every 40 to 50 clocks: up to 64 tokens two warps issue, stage `it` going to issuer it % 2, each into
     // an accumulator of its own (added up in the epilogue).  A parity wait is only safe on consecutive phases, so every
     // barrier must always be waited on by the same thread or group: the ring lengths are multiples of the issuer count
     // and of the number of decode groups (each group then owns two A slots and every other packed slot).  With one
     // issuer the A ring may have three slots although the groups then share them: a group that waits for the release of
     // use u of a slot (stage it) has, for the stage it stored before (it - 1 or it - 3), already waited for an MMA no
     // earlier than it - 6, the one that ended use u - 2; MMAs complete in order, so the wait is on the next phase.
-    static constexpr int kIssuers = BN <= 32 ? 2 : 1;
+    static constexpr int kIssuers = BN <= 64 ? 2 : 1;
     static constexpr int kSA = kIssuers == 2 ? 4 : 3;
-    static constexpr int kSB = BN <= 16 ? 8 : (BN <= 32 ? (K <= 3 ? 6 : 4) : (BN <= 64 ? 4 : 2));
+    static constexpr int kSB = BN <= 16 ? 8 : (BN <= 32 ? (K <= 3 ? 6 : 4) : 2);
     static constexpr int kRest = kSmemBudget - kSA * kATileBytes - kSB * kBTileBytes - 2048;
     static constexpr int kSP = (kRest / kBlockBytes > 8 ? 8 : kRest / kBlockBytes) / kDecodeGroups * kDecodeGroups;
     static_assert(kSP >= 2, "at least two packed blocks in flight");
