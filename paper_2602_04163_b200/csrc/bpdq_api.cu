@@ -162,7 +162,10 @@ extern "C" int bpdq_create(bpdq_handle_t* hp, int out, int in, int K, int group,
     // against 64 us for two look-up-table passes and 67-78 us for the tcgen05 tile kernel); from 17 tokens on its second
     // token tile costs more than the tile kernel.
     h->few_max_m = 16;
-    if (K == 4) { h->gemv_max_m = 4; h->few_max_m = 0; }   // sixteen candidates: the few-token kernel's decode no longer fits its registers (110 us), two look-up-table passes do better
+    // sixteen candidates (the few-token kernel then takes tasks of two row groups): 83-88 us on the largest projections for
+    // 3 to 16 tokens against 77 / 92 us for two look-up-table passes at 3 / 4 tokens (103 / 120 us at g = 64) and 118 us
+    // for the tile kernel
+    if (K == 4) h->gemv_max_m = group == 64 ? 2 : 3;
 
     const size_t stage_x = (size_t)max_M * in * 2, stage_y = (size_t)max_M * out * 2;
     if ((e = cudaMalloc(&h->d_blob, h->blob_bytes)) != cudaSuccess ||

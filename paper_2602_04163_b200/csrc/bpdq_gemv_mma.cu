@@ -52,6 +52,8 @@ constexpr int kMiscBytes = 4096;                      // completion list, abort 
 constexpr int kMaxDone = 512;
 constexpr int kMaxBatch = BPDQ_BATCH_MAX;
 constexpr int kMaxGrid = 192;
+// eight-row groups per task: four, or two with sixteen candidates per group (K = 4), whose units and tables would not fit the registers otherwise
+template <int K> constexpr int kRowGroups = K == 4 ? 2 : 4;
 constexpr int kSegmentCost = 2;                       // staging the activations of a segment, in (row group x column range) tasks
 
 struct MmaLinear {
@@ -534,12 +536,13 @@ int launch_k(bpdq_handle_s* h, const MmaParams& p, cudaStream_t stream) {
     const bool g64 = p.lin[0].group == 64;
     bool ext = false;
     for (int k = 0; k < p.n; ++k) ext = ext || p.lin[k].bias_a || p.lin[k].conv_b;
+    constexpr int NJ = kRowGroups<K>;
     if (p.M <= 16) {
-        if (ext) return g64 ? launch_cfg<K, 1, true, 4, 16, true>(h, p, stream) : launch_cfg<K, 1, false, 4, 16, true>(h, p, stream);
-        return g64 ? launch_cfg<K, 1, true, 4, 16, false>(h, p, stream) : launch_cfg<K, 1, false, 4, 16, false>(h, p, stream);
+        if (ext) return g64 ? launch_cfg<K, 1, true, NJ, 16, true>(h, p, stream) : launch_cfg<K, 1, false, NJ, 16, true>(h, p, stream);
+        return g64 ? launch_cfg<K, 1, true, NJ, 16, false>(h, p, stream) : launch_cfg<K, 1, false, NJ, 16, false>(h, p, stream);
     }
-    if (ext) return g64 ? launch_cfg<K, 2, true, 4, 16, true>(h, p, stream) : launch_cfg<K, 2, false, 4, 16, true>(h, p, stream);
-    return g64 ? launch_cfg<K, 2, true, 4, 16, false>(h, p, stream) : launch_cfg<K, 2, false, 4, 16, false>(h, p, stream);
+    if (ext) return g64 ? launch_cfg<K, 2, true, NJ, 16, true>(h, p, stream) : launch_cfg<K, 2, false, NJ, 16, true>(h, p, stream);
+    return g64 ? launch_cfg<K, 2, true, NJ, 16, false>(h, p, stream) : launch_cfg<K, 2, false, NJ, 16, false>(h, p, stream);
 }
 
 }  // namespace
@@ -563,7 +566,7 @@ int few_prepare(bpdq_handle_s* h) {
     const int K = h->K;
     const int ngs = 512 / h->group;
     alignas(64) CUtensorMap maps[2];
-    constexpr int rows = 32;                                              // a task: four groups of eight rows
+    const int rows = K == 4 ? 16 : 32;                                    // a task: four groups of eight rows (two at K = 4)
     const cuuint32_t estr3[3] = {1, 1, 1};
     const cuuint64_t pd[3] = {16, (cuuint64_t)(h->in / 128) * K, (cuuint64_t)h->out / 8};
     const cuuint64_t ps[2] = {(cuuint64_t)h->out * 16, 128};

@@ -26,6 +26,8 @@ pytestmark = pytest.mark.gpu
     (4, 64, 48, 1536, 11),
     (1, 64, 1024, 2048, 2),
     (2, 128, 1040, 8192, 16),     # sixteen slices: four column ranges accumulate through the workspace
+    (4, 128, 2064, 2048, 16),     # sixteen candidates with tasks of two row groups: several segments per CTA, ragged last task
+    (4, 64, 1040, 4096, 20),      # the same with two token tiles and a coefficient group per half block
 ])
 def test_few_token_kernel(K, g, out, in_, M):
     h, bits, coef = G.make_layer(140 + K, out, in_, K, g, max_M=M)
@@ -55,7 +57,7 @@ def test_few_token_kernel_multiplies_the_dequantized_weights(K):
 
 
 @pytest.mark.parametrize("name,out,in_,K,M", [("gate", 29568, 8192, 2, 16), ("down", 8192, 29568, 3, 8), ("gate", 29568, 8192, 3, 32),
-                                               ("down", 8192, 29568, 2, 5), ("7b_down", 3584, 18944, 2, 16)])
+                                               ("down", 8192, 29568, 2, 5), ("7b_down", 3584, 18944, 2, 16), ("gate", 29568, 8192, 4, 12)])
 def test_few_token_kernel_full_size_sampled(name, out, in_, K, M):
     """Benchmark-sized layers generated on the device; sampled rows against the checker."""
     g = 128
