@@ -10,8 +10,8 @@
 //
 //   D[token, row] (16 x 8) += A[token, k] (16 x 16, activations) * B[k, row] (16 x 8, decoded weights)
 //
-// Work split.  A warp task is 32 output rows x 512 input columns (a "slice" of four 128-column blocks): lane
-// (g, t) = (lane / 4, lane % 4) owns the rows 8j + g (j = 0..3) of block t.  The task's packed bytes -- 4 K runs of
+// Work split.  A warp task is 16 output rows x 512 input columns (a "slice" of four 128-column blocks): lane
+// (g, t) = (lane / 4, lane % 4) owns the rows 8j + g (j = 0, 1) of block t.  The task's packed bytes -- 4 K runs of
 // 512 bytes of plane units and a few 64-byte runs of binary16 coefficients -- arrive one task ahead in the warp's
 // private landing area in shared memory as two boxes of tensor maps over the blob (two TMA copies per task whatever
 // K is, completion on the warp's mbarrier; per-lane 16-byte asynchronous copies of the same bytes cost one
@@ -23,7 +23,7 @@
 // registers of two binary16 each -- exactly the B fragments of two mma.sync instructions.  The k index of an
 // instruction is ours to assign: lane t supplies four consecutive columns of ITS block, so one instruction
 // contracts 4 blocks x 4 columns, and the activations are staged in shared memory in that order, already cut
-// into A fragments (one 16-byte load per lane and instruction, shared by the four row groups of the task).
+// into A fragments (one 16-byte load per lane and instruction, shared by the two row groups of the task).
 // Accumulators stay in registers while a warp walks along the columns of one row group and leave as binary32
 // atomic adds into the handle's workspace [token][row]; arrival counters per 128 rows tell the CTA that
 // delivers the last contribution to round those rows to binary16, write y and zero the workspace again
@@ -52,8 +52,9 @@ constexpr int kMiscBytes = 4096;                      // completion list, abort 
 constexpr int kMaxDone = 512;
 constexpr int kMaxBatch = BPDQ_BATCH_MAX;
 constexpr int kMaxGrid = 192;
-// eight-row groups per task: four, or two with sixteen candidates per group (K = 4), whose units and tables would not fit the registers otherwise
-template <int K> constexpr int kRowGroups = K == 4 ? 2 : 4;
+// Eight-row groups per task.  Two: with four, the units and tables of sixteen candidates per group (K = 4) do not fit the
+// registers, and the other K ran 2 to 20 % slower (most with two token tiles).
+constexpr int kRowGroups = 2;
 constexpr int kSegmentCost = 2;                       // staging the activations of a segment, in (row group x column range) tasks
 
 struct MmaLinear {
@@ -529,14 +530,14 @@ int launch_cfg(bpdq_handle_s* h, MmaParams p, cudaStream_t stream) {
     return BPDQ_OK;
 }
 
-// Four row groups per task and sixteen warps: eight warps with twice the registers, or 24 to 32 warps on tasks of two
-// row groups, ran within 5 % of this (the kernel is bound by the instruction pipes, not by latency).
+// Sixteen warps: eight warps with twice the registers, or 24 to 32 warps with fewer, ran within 5 % of this (the kernel is
+// bound by the instruction pipes, not by latency).
 template <int K>
 int launch_k(bpdq_handle_s* h, const MmaParams& p, cudaStream_t stream) {
     const bool g64 = p.lin[0].group == 64;
     bool ext = false;
     for (int k = 0; k < p.n; ++k) ext = ext || p.lin[k].bias_a || p.lin[k].conv_b;
-    constexpr int NJ = kRowGroups<K>;
+    constexpr int NJ = kRowGroups;
     if (p.M <= 16) {
         if (ext) return g64 ? launch_cfg<K, 1, true, NJ, 16, true>(h, p, stream) : launch_cfg<K, 1, false, NJ, 16, true>(h, p, stream);
         return g64 ? launch_cfg<K, 1, true, NJ, 16, false>(h, p, stream) : launch_cfg<K, 1, false, NJ, 16, false>(h, p, stream);
@@ -556,7 +557,7 @@ bool gemv_mma_supported(int out, int in, int K, int group) {
 
 // Tensor maps of a handle's blob for this kernel's two copies per task, encoded on the host and kept in device
 // memory: plane units as (128 bytes = eight rows) x (block, plane) x (eight-row group), coefficients as rows (group,
-// coefficient) of out x 2 bytes, both in 8-byte elements; boxes of one task (32 output rows x one 512-column
+// coefficient) of out x 2 bytes, both in 8-byte elements; boxes of one task (16 output rows x one 512-column
 // slice).  Leaves d_few_maps null (and the kernel unavailable for this handle)
 // when the driver has no encoder.
 int few_prepare(bpdq_handle_s* h) {
@@ -566,7 +567,7 @@ int few_prepare(bpdq_handle_s* h) {
     const int K = h->K;
     const int ngs = 512 / h->group;
     alignas(64) CUtensorMap maps[2];
-    const int rows = K == 4 ? 16 : 32;                                    // a task: four groups of eight rows (two at K = 4)
+    constexpr int rows = 8 * kRowGroups;                                  // output rows of a task
     const cuuint32_t estr3[3] = {1, 1, 1};
     const cuuint64_t pd[3] = {16, (cuuint64_t)(h->in / 128) * K, (cuuint64_t)h->out / 8};
     const cuuint64_t ps[2] = {(cuuint64_t)h->out * 16, 128};
