@@ -149,7 +149,7 @@ BPDQ_API int bpdq_dequant(bpdq_handle_t h, void* w_fp16_dev, void* stream);
 /* The quantized linear map y = x * W^T (paper: Eq. 1 applied to activations, Section 3.1).
  * x: device binary16 [M][in]; y: device binary16 [M][out]; 0 <= M <= max_M.  M == 0 returns
  * BPDQ_OK without a launch.  Picks the look-up-table kernel for the smallest M (default: up to
- * 2 tokens), the few-token kernel above that (default: up to 16 tokens) and the tcgen05 kernel
+ * 2 tokens, 3 at K = 4 and g >= 128), the few-token kernel above that (default: up to 16 tokens) and the tcgen05 kernel
  * beyond (also below when the packed weights of the linear reach 4 GB, which the look-up-table
  * kernel's 32-bit offsets do not cover).  x and y must not alias. */
 BPDQ_API int bpdq_linear(bpdq_handle_t h, const void* x_fp16_dev, void* y_fp16_dev, int M, void* stream);
