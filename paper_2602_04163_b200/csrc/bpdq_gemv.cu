@@ -158,6 +158,16 @@ __device__ __forceinline__ void lookup2_add(unsigned long long& acc, unsigned ad
         "add.rn.f32x2 %0, %0, t;\n\t}"
         : "+l"(acc) : "r"(addr0), "r"(addr1), "n"(IMM0), "n"(IMM1));
 }
+// The same, and the two loaded values are handed back (g = 64 adds them to the first group's partial sums as well).
+template <int IMM0, int IMM1>
+__device__ __forceinline__ void lookup2v_add(unsigned long long& acc, unsigned addr0, unsigned addr1, float& a, float& b) {
+    asm("{\n\t.reg .b64 t;\n\t"
+        "ld.shared.f32 %1, [%3+%5];\n\t"
+        "ld.shared.f32 %2, [%4+%6];\n\t"
+        "mov.b64 t, {%1, %2};\n\t"
+        "add.rn.f32x2 %0, %0, t;\n\t}"
+        : "+l"(acc), "=&f"(a), "=&f"(b) : "r"(addr0), "r"(addr1), "n"(IMM0), "n"(IMM1));
+}
 __device__ __forceinline__ float2 unpack2(unsigned long long v) {
     float2 f;
     asm("mov.b64 {%0, %1}, %2;" : "=f"(f.x), "=f"(f.y) : "l"(v));
@@ -463,25 +473,26 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_lut_kernel(const __grid_consta
                         addr[i] = prmt(word_of(tk.pl[q][i], st >> 2), slots[st / 3], 0xC400u | ((st & 3) << 4) | (5 + st % 3));   // the selector is a constant once the step loop is unrolled
                     constexpr int QI = 128;               // the block pair and the token's table go into the immediate
                     if constexpr (G64) {
-                        float v[NS];
+                        // pairs as below (two planes of one token, or the two tokens of a plane); the loaded values also go, on
+                        // the steps of the block's first 64 columns, into the first group's partial sums
+                        const bool lo = ((lo_steps >> st) & 1u) != 0u;
 #pragma unroll
-                        for (int i = 0; i < K; ++i)
-#pragma unroll
-                            for (int m = 0; m < MT; ++m) {
-                                if (m == 0 && q == 0) v[i * MT + m] = lds_table<0>(addr[i]);
-                                else if (m == 0) v[i * MT + m] = lds_table<QI>(addr[i]);
-                                else if (q == 0) v[i * MT + m] = lds_table<kTableBytes>(addr[i]);
-                                else v[i * MT + m] = lds_table<kTableBytes + QI>(addr[i]);
+                        for (int j = 0; j < NS / 2; ++j) {
+                            float va, vb;
+                            if constexpr (MT == 2) {
+                                if (q == 0) lookup2v_add<0, kTableBytes>(acc[j][st & 1], addr[j], addr[j], va, vb);
+                                else lookup2v_add<QI, kTableBytes + QI>(acc[j][st & 1], addr[j], addr[j], va, vb);
+                            } else {
+                                if (q == 0) lookup2v_add<0, 0>(acc[j][st & 1], addr[2 * j], addr[2 * j + 1], va, vb);
+                                else lookup2v_add<QI, QI>(acc[j][st & 1], addr[2 * j], addr[2 * j + 1], va, vb);
                             }
-                        if ((lo_steps >> st) & 1u) {
-#pragma unroll
-                            for (int j = 0; j < NS; ++j) Slo[j] += v[j];
+                            if (lo) { Slo[2 * j] += va; Slo[2 * j + 1] += vb; }
                         }
-#pragma unroll
-                        for (int j = 0; j < NS / 2; ++j) add2(acc[j][st & 1], v[2 * j], v[2 * j + 1]);
-                        if (NS & 1) {
-                            if ((st & 1) == 0) held = v[NS - 1];
-                            else add2(acc[NP - 1][(st >> 1) & 1], held, v[NS - 1]);
+                        if (NS & 1) {                     // one token, odd K: the last plane pairs two consecutive steps
+                            const float vl = q == 0 ? lds_table<0>(addr[K - 1]) : lds_table<QI>(addr[K - 1]);
+                            if (lo) Slo[NS - 1] += vl;
+                            if ((st & 1) == 0) held = vl;
+                            else add2(acc[NP - 1][(st >> 1) & 1], held, vl);
                         }
                     } else if constexpr (MT == 2) {
                         // pair = the two tokens of one plane: one address, two tables
