@@ -228,6 +228,25 @@ class Layer:
             h.bpdq_destroy()
 
 
+def graph_replay_ms(torch, binding, stream, layers, groups, xs, ys, n):
+    """Records the batched launches of every layer copy (M = 1) into one CUDA graph and times n layers' worth of replays."""
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for hs in layers:
+            for grp in groups:
+                binding.bpdq_linear_batch([hs[j] for j in grp], [xs[hs[j].in_].data_ptr() for j in grp], [ys[j].data_ptr() for j in grp],
+                                          1, side.cuda_stream)
+    replays = max(1, n // len(layers))
+
+    def run():
+        for _ in range(replays):
+            graph.replay()
+    run()
+    return event_time_ms(torch, run, stream) * n / (replays * len(layers))
+
+
 def event_time_ms(torch, fn, stream):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
@@ -513,6 +532,10 @@ def extra_sections(torch, binding, args, peaks, sp, stream):
             out[f"gemv_layer_batched_{label}_K{K}"] = {"launches_per_layer": len(groups), "us_per_layer": ms * 1e3,
                                                        "gbs": b / (ms * 1e-3) / 1e9, "frac_measured": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                                        "l2": f"{copies} layer copies of {b / 1e6:.0f} MB rotated"}
+            if label == "decoder_groups":
+                # the same launches recorded once into a CUDA graph (all copies, so that the rotation stays) and replayed
+                ms_g = graph_replay_ms(torch, binding, stream, layers, groups, xs, ys, n) / n
+                out[f"gemv_layer_batched_{label}_K{K}"]["cuda_graph_us_per_layer"] = ms_g * 1e3
         for L in layers:
             for h in L:
                 h.bpdq_destroy()
@@ -536,6 +559,20 @@ def extra_sections(torch, binding, args, peaks, sp, stream):
         out[f"gemv_layer_7b_batched_K{K}"] = {"launches_per_layer": 1, "us_per_layer": ms * 1e3, "gbs": b / (ms * 1e-3) / 1e9,
                                               "frac_measured": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                               "l2": f"{copies} layer copies of {b / 1e6:.0f} MB rotated"}
+        # the grouping a decoder allows, as direct calls and as a replayed CUDA graph (small launches: here the host's
+        # launch cost shows)
+        groups7b = [[0, 1, 2], [3], [4, 5], [6]]
+
+        def run_7b_groups():
+            for k in range(n):
+                hs = layers[k % copies]
+                for grp in groups7b:
+                    binding.bpdq_linear_batch([hs[j] for j in grp], [xs[hs[j].in_].data_ptr() for j in grp], [ys[j].data_ptr() for j in grp], 1, sp)
+        run_7b_groups()
+        ms_d = event_time_ms(torch, run_7b_groups, stream) / n
+        ms_g = graph_replay_ms(torch, binding, stream, layers, groups7b, xs, ys, n) / n
+        out[f"gemv_layer_7b_decoder_groups_K{K}"] = {"launches_per_layer": 4, "us_per_layer": ms_d * 1e3, "cuda_graph_us_per_layer": ms_g * 1e3,
+                                                    "gbs": b / (ms_d * 1e-3) / 1e9, "frac_measured": b / (ms_d * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         for L in layers:
             for h in L:
                 h.bpdq_destroy()
