@@ -31,6 +31,12 @@
  *     serialised by the caller; calls on different handles may run concurrently from
  *     different threads.  A handle is used with the device that was current when it was
  *     created: calling with another current device is BPDQ_ERR_INVALID, nothing is launched;
+ *   - stream capture: once a handle has run a given kind of call outside a capture (its first use
+ *     sets shared-memory limits, launch plans and tensor maps), bpdq_dequant, bpdq_linear,
+ *     bpdq_linear_ex, bpdq_linear_batch and bpdq_gate_up_swiglu only enqueue kernels on `stream`
+ *     (no allocation, no copy, no host wait) and may be recorded into a CUDA graph; x, y and the
+ *     handles must then stay where they are for the replays.  The *_host calls, bpdq_get_status
+ *     and bpdq_read_blob wait for the stream and cannot be recorded;
  *   - supported shapes: K in {1,2,3,4}; g in {64,128,256}; in % 128 == 0 and in % g == 0;
  *     out % 16 == 0.  Anything else is BPDQ_ERR_UNSUPPORTED.
  *
