@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 LAYER = [("q", 512, 512), ("k", 128, 512), ("v", 128, 512), ("o", 512, 512), ("gate", 1408, 512), ("up", 1408, 512), ("down", 512, 1408)]
 
 
-def _enqueue_layer(hs, x_hidden, x_inter, ys, h_unit, M, sp):
+def _enqueue_layer(hs, x_hidden, x_inter, ys, h_unit, w_q, M, sp):
     """The launches a decoder issues for its seven projections: {q, k, v}, {o}, the gated unit over {gate, up}, {down}.
     (Attention and the residual adds are not part of this library: o and down read given activations.)"""
     if M <= binding.GEMV_MAX_M:
@@ -27,6 +27,7 @@ def _enqueue_layer(hs, x_hidden, x_inter, ys, h_unit, M, sp):
     hs[3].bpdq_linear(x_hidden.data_ptr(), ys[3].data_ptr(), M, sp)
     binding.bpdq_gate_up_swiglu(hs[4], hs[5], x_hidden.data_ptr(), h_unit.data_ptr(), M, sp)
     hs[6].bpdq_linear(x_inter.data_ptr(), ys[6].data_ptr(), M, sp)
+    hs[0].bpdq_dequant(w_q.data_ptr(), sp)               # not a decoder's step; recorded to show that it can be
 
 
 @pytest.mark.parametrize("K,M", [(2, 1), (3, 2), (2, 8), (3, 40), (2, 300)])
@@ -40,6 +41,7 @@ def test_decoder_layer_as_a_cuda_graph(K, M):
     x_inter = torch.zeros((M, 1408), dtype=torch.float16, device="cuda")
     ys = [torch.zeros((M, o), dtype=torch.float16, device="cuda") for _, o, _ in LAYER]
     h_unit = torch.zeros((M, 1408), dtype=torch.float16, device="cuda")
+    w_q = torch.zeros((512, 512), dtype=torch.float16, device="cuda")
 
     def load(seed):
         xh, xi = synth.activations(seed, M, 512), synth.activations(seed + 1, M, 1408)
@@ -50,18 +52,19 @@ def test_decoder_layer_as_a_cuda_graph(K, M):
     # first use outside the capture: shared-memory opt-ins, launch plans and tensor maps are set up once per handle
     load(810)
     with torch.cuda.stream(stream):
-        _enqueue_layer(hs, x_hidden, x_inter, ys, h_unit, M, sp)
+        _enqueue_layer(hs, x_hidden, x_inter, ys, h_unit, w_q, M, sp)
     stream.synchronize()
 
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph, stream=stream):
-        _enqueue_layer(hs, x_hidden, x_inter, ys, h_unit, M, sp)
+        _enqueue_layer(hs, x_hidden, x_inter, ys, h_unit, w_q, M, sp)
 
     for seed in (820, 830):                              # two replays, each on new activations in the captured buffers
         xh, xi = load(seed)
         for y in ys:
             y.fill_(float("nan"))
         h_unit.fill_(float("nan"))
+        w_q.zero_()
         torch.cuda.synchronize()
         graph.replay()
         torch.cuda.synchronize()
@@ -82,5 +85,6 @@ def test_decoder_layer_as_a_cuda_graph(K, M):
         silu_g = oracle.swiglu(yg, np.ones_like(yg))
         bound = 1.1 * (np.abs(yu) + du) * dg + (np.abs(silu_g) + 1.1 * dg) * du + 2.0 ** -10 * np.abs(h_ref) + 1e-4
         assert np.all(np.abs(got - h_ref) <= bound), f"replayed gated unit seed {seed}"
+        assert np.array_equal(w_q.view(torch.int16).cpu().numpy().view(np.uint16), oracle.dequant(layers[0][1], layers[0][2], g))
     for h in hs:
         h.bpdq_destroy()
