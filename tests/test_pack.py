@@ -57,6 +57,29 @@ def test_bits_per_weight_matches_table_1(golden_dir):
         assert abs(bpw - float(printed)) <= 0.005 + 1e-12   # the table rounds to two decimals
 
 
+def test_model_sizes_match_the_printed_ones(golden_dir):
+    """Storage accounting at model level: decoder-layer linears in the packed format (K/8 + 2 (K+1)/g bytes per weight,
+    cross-checked against bpdq_packed_bytes where the library takes the shape), embedding and head in binary16."""
+    models = {"7b": (synth.QWEN25_7B_LAYER, 28, 3584), "72b": (synth.QWEN25_72B_LAYER, 80, 8192)}
+    vocab = 152064
+    rows = [ln.split() for ln in open(f"{golden_dir}/model_size_gib.txt") if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 7
+    for model, K, g, printed in rows:
+        layer, n_layers, hidden = models[model]
+        K, g, printed = int(K), int(g), float(printed)
+        if K == 16:
+            layer_bytes = sum(2 * o * i for _, o, i in layer)
+        else:
+            layer_bytes = sum(o * i * K // 8 + o * i * 2 * (K + 1) // g for _, o, i in layer)
+            if all(i % g == 0 for _, _, i in layer):
+                assert layer_bytes == sum(binding.bpdq_packed_bytes(o, i, K, g) for _, o, i in layer)
+        gib = (n_layers * layer_bytes + 2 * vocab * hidden * 2) / 2 ** 30
+        # the 7B rows agree to the table's two decimals; the 72B figure (norm weights and whatever else the checkpoint
+        # holds are not counted here) to one per cent
+        tol = 0.0075 if model == "7b" else 0.01 * printed
+        assert abs(gib - printed) <= tol, (model, K, g, gib, printed)
+
+
 def test_workload_byte_counts():
     """Useful bytes of the benchmark layers (planes + binary16 coefficients, g = 128)."""
     assert binding.bpdq_packed_bytes(4096, 4096, 2, 128) == 4_980_736
