@@ -70,11 +70,11 @@ def float_to_half(f: float) -> int:
 
 
 def dequant(bits: np.ndarray, coef: np.ndarray, group: int) -> np.ndarray:
-    """bits uint8 [K][out][in], coef uint16 [K+1][out][in/group] -> fp16 bit patterns uint16 [out][in]."""
+    """bits uint8 [K][out][in], coef uint16 [K+1][out][ceil(in/group)] -> fp16 bit patterns uint16 [out][in]."""
     bits = _c(bits, np.uint8)
     coef = _c(coef, np.uint16)
     K, out, in_ = bits.shape
-    assert coef.shape == (K + 1, out, in_ // group), (coef.shape, bits.shape, group)
+    assert coef.shape == (K + 1, out, -(-in_ // group)), (coef.shape, bits.shape, group)
     w = np.empty((out, in_), dtype=np.uint16)
     rc = _load().oracle_dequant(_ptr(bits), _ptr(coef), out, in_, K, group, _ptr(w))
     if rc:
@@ -90,7 +90,7 @@ def linear(bits: np.ndarray, coef: np.ndarray, x: np.ndarray, group: int):
     K, out, in_ = bits.shape
     M = x.shape[0]
     assert x.shape == (M, in_)
-    assert coef.shape == (K + 1, out, in_ // group)
+    assert coef.shape == (K + 1, out, -(-in_ // group))
     y = np.empty((M, out), dtype=np.float64)
     a = np.empty((M, out), dtype=np.float64)
     rc = _load().oracle_linear(_ptr(bits), _ptr(coef), _ptr(x), out, in_, K, group, M, _ptr(y), _ptr(a))
@@ -100,12 +100,12 @@ def linear(bits: np.ndarray, coef: np.ndarray, x: np.ndarray, group: int):
 
 
 def unpack(blob: np.ndarray, out: int, in_: int, K: int, group: int):
-    """Device blob (uint8) -> (bits uint8 [K][out][in], coef uint16 [K+1][out][in/group])."""
+    """Device blob (uint8) -> (bits uint8 [K][out][in], coef uint16 [K+1][out][ceil(in/group)])."""
     blob = _c(blob, np.uint8)
-    need = out * in_ * K // 8 + out * (in_ // group) * (K + 1) * 2
+    need = out * in_ * K // 8 + out * (-(-in_ // group)) * (K + 1) * 2
     assert blob.size == need, (blob.size, need)
     bits = np.empty((K, out, in_), dtype=np.uint8)
-    coef = np.empty((K + 1, out, in_ // group), dtype=np.uint16)
+    coef = np.empty((K + 1, out, -(-in_ // group)), dtype=np.uint16)
     rc = _load().oracle_unpack(_ptr(blob), out, in_, K, group, _ptr(bits), _ptr(coef))
     if rc:
         raise ValueError("oracle_unpack rejected its arguments")

@@ -9,6 +9,9 @@
 // What it follows:
 //   * Variable grid (Methodology, Eq. 1):  W^[r,j] = C0[r,G] + sum_{i=1..K} Ci[r,G] * Bi[r,j],
 //     Bi in {0,1}, G = floor(j / g)  (REP repeats a group coefficient over its g columns).
+//     Where `in` is not a multiple of g the last group holds the remaining columns: the paper runs
+//     g = 256 on a model whose down projection has 115.5 x 256 input channels and does not say how;
+//     G = floor(j / g) needs no more than ceil(in / g) coefficient groups per row.
 //   * Candidate values of a group (Eq. 7; Appendix A.2: {0, c1, c2, c1+c2} for K = 2).
 //   * Quantized linear map (Section 3.1): the layer output is W^ applied to the activations,
 //     per token  y[m,r] = sum_j x[m,j] * W^[r,j].
@@ -130,11 +133,11 @@ extern "C" {
 float oracle_half_to_float(uint16_t h) { return half_bits_to_float(h); }
 uint16_t oracle_float_to_half(float f) { return float_to_half_bits(f); }
 
-// bits [K][out][in] (0/1), coef [K+1][out][in/g] fp16 bits -> w [out][in] fp16 bits.
+// bits [K][out][in] (0/1), coef [K+1][out][ceil(in/g)] fp16 bits -> w [out][in] fp16 bits.
 int oracle_dequant(const uint8_t* bits, const uint16_t* coef, int64_t out, int64_t in, int K,
                    int64_t g, uint16_t* w) {
-    if (!bits || !coef || !w || out <= 0 || in <= 0 || K < 1 || g <= 0 || in % g) return 1;
-    const int64_t ngroups = in / g;
+    if (!bits || !coef || !w || out <= 0 || in <= 0 || K < 1 || g <= 0) return 1;
+    const int64_t ngroups = (in + g - 1) / g;          // the last group may be short
     for (int64_t r = 0; r < out; ++r)
         for (int64_t j = 0; j < in; ++j)
             w[r * in + j] = decode_one(bits, coef, out, in, K, ngroups, r, j, j / g);
@@ -144,9 +147,9 @@ int oracle_dequant(const uint8_t* bits, const uint16_t* coef, int64_t out, int64
 // x [M][in] fp16 bits -> y [M][out], a [M][out] in binary64 (a may be NULL).
 int oracle_linear(const uint8_t* bits, const uint16_t* coef, const uint16_t* x, int64_t out,
                   int64_t in, int K, int64_t g, int64_t M, double* y, double* a) {
-    if (!bits || !coef || !x || !y || out <= 0 || in <= 0 || K < 1 || g <= 0 || in % g || M < 0)
+    if (!bits || !coef || !x || !y || out <= 0 || in <= 0 || K < 1 || g <= 0 || M < 0)
         return 1;
-    const int64_t ngroups = in / g;
+    const int64_t ngroups = (in + g - 1) / g;          // the last group may be short
     for (int64_t r = 0; r < out; ++r) {
         for (int64_t m = 0; m < M; ++m) { y[m * out + r] = 0.0; if (a) a[m * out + r] = 0.0; }
         for (int64_t j = 0; j < in; ++j) {
@@ -170,7 +173,7 @@ int oracle_linear(const uint8_t* bits, const uint16_t* coef, const uint16_t* x, 
 // function unchanged.  perm must be a permutation of 0..in-1 (checked).
 int oracle_linear_perm(const uint8_t* bits, const uint16_t* coef, const uint16_t* x, const int64_t* perm, int64_t out,
                        int64_t in, int K, int64_t g, int64_t M, double* y, double* a) {
-    if (!bits || !coef || !x || !perm || !y || out <= 0 || in <= 0 || K < 1 || g <= 0 || in % g || M < 0) return 1;
+    if (!bits || !coef || !x || !perm || !y || out <= 0 || in <= 0 || K < 1 || g <= 0 || M < 0) return 1;
     {
         uint8_t* seen = new uint8_t[in]();
         bool ok = true;
@@ -181,7 +184,7 @@ int oracle_linear_perm(const uint8_t* bits, const uint16_t* coef, const uint16_t
         delete[] seen;
         if (!ok) return 1;
     }
-    const int64_t ngroups = in / g;
+    const int64_t ngroups = (in + g - 1) / g;          // the last group may be short
     for (int64_t r = 0; r < out; ++r) {
         for (int64_t m = 0; m < M; ++m) { y[m * out + r] = 0.0; if (a) a[m * out + r] = 0.0; }
         for (int64_t j = 0; j < in; ++j) {
@@ -216,9 +219,9 @@ int oracle_add_bias(double* y, const uint16_t* bias, int64_t M, int64_t out) {
 // Device blob -> logical tensors (layout described in the header comment of this file).
 int oracle_unpack(const uint8_t* blob, int64_t out, int64_t in, int K, int64_t g, uint8_t* bits,
                   uint16_t* coef) {
-    if (!blob || !bits || !coef || out <= 0 || in <= 0 || K < 1 || g <= 0 || in % g || in % 128)
+    if (!blob || !bits || !coef || out <= 0 || in <= 0 || K < 1 || g <= 0 || in % 128)
         return 1;
-    const int64_t nblocks = in / 128, ngroups = in / g;
+    const int64_t nblocks = in / 128, ngroups = (in + g - 1) / g;
     for (int64_t b = 0; b < nblocks; ++b)
         for (int i = 0; i < K; ++i)
             for (int64_t r = 0; r < out; ++r) {
