@@ -53,7 +53,7 @@ TIMED_BLOCKS = 25
 
 def useful_bytes(out: int, in_: int, K: int, g: int, M: int) -> int:
     """Algorithmic HBM bytes of one linear call: packed planes + binary16 coefficients + x + y."""
-    return out * in_ * K // 8 + out * (in_ // g) * (K + 1) * 2 + M * in_ * 2 + M * out * 2
+    return out * in_ * K // 8 + out * (-(-in_ // g)) * (K + 1) * 2 + M * in_ * 2 + M * out * 2    # ceil(in / g) groups: a last one may be short
 
 
 def layer_bytes(shapes, K: int, M: int) -> int:
@@ -634,7 +634,7 @@ def extra_sections(torch, binding, args, peaks, sp, stream):
     # the paper's own formats (Table 1) on the 72B-shaped layer: decode as one batched launch, prefill at M = 8192
     for tag, K, g in (("W2-G64", 2, 64), ("W3-G64", 3, 64), ("W2-G256", 2, 256), ("W4-G128", 4, 128)):
         copies = 3
-        gof = lambda i: g if i % g == 0 else 128      # 29568 input columns are not a multiple of 256: that linear keeps groups of 128
+        gof = lambda i: g                             # 29568 input columns are 115.5 groups of 256: the last group of a row is short
         layers = [[binding.Handle(o, i, K, gof(i), None, 1100 + 10 * c + li, 1) for li, (_, o, i) in enumerate(shapes)] for c in range(copies)]
         xs1 = {8192: xt(1, 8192), 29568: xt(1, 29568)}
         ys1 = [torch.empty((1, o), dtype=torch.float16, device="cuda") for _, o, _ in shapes]

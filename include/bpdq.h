@@ -37,12 +37,14 @@
  *     (no allocation, no copy, no host wait) and may be recorded into a CUDA graph; x, y and the
  *     handles must then stay where they are for the replays.  The *_host calls, bpdq_get_status
  *     and bpdq_read_blob wait for the stream and cannot be recorded;
- *   - supported shapes: K in {1,2,3,4}; g in {64,128,256}; in % 128 == 0 and in % g == 0;
- *     out % 16 == 0.  Anything else is BPDQ_ERR_UNSUPPORTED.
+ *   - supported shapes: K in {1,2,3,4}; g in {64,128,256}; in % 128 == 0; out % 16 == 0.  Anything
+ *     else is BPDQ_ERR_UNSUPPORTED.  With g = 256 and in % 256 == 128 the last group of a row holds the
+ *     remaining 128 columns (ceil(in/g) groups per row; the paper applies g = 256 to a 29568-channel input
+ *     and does not say how); the host producers take whole groups only.
  *
  * Logical tensors (what pack/unpack exchange with the caller)
  *   bits : uint8  [K][out][in], values 0/1; bits[i] is the paper's plane B_{i+1}
- *   coef : uint16 [K+1][out][in/g], binary16 bit patterns; coef[0] is C0, coef[i] is Ci
+ *   coef : uint16 [K+1][out][ceil(in/g)], binary16 bit patterns; coef[0] is C0, coef[i] is Ci
  *
  * Packed blob (what lives in device memory), bpdq_packed_bytes() bytes, no padding:
  *   planes, then coefficients.
@@ -105,7 +107,7 @@ enum {
 #define BPDQ_NOALLOC_MAX_OUT 65536   /* most output rows bpdq_linear_noalloc accepts */
 
 /* Storage accounting (paper: Table 1, column BPW = K + 16 (K+1) / g bits per weight).
- * Bytes of the packed blob: out*in*K/8 + out*(in/g)*(K+1)*2.  Returns 0 for an unsupported
+ * Bytes of the packed blob: out*in*K/8 + out*ceil(in/g)*(K+1)*2.  Returns 0 for an unsupported
  * shape.  Host only, no CUDA call. */
 BPDQ_API size_t bpdq_packed_bytes(int out, int in, int K, int group);
 

@@ -94,11 +94,11 @@ def bpdq_packed_bytes(out: int, in_: int, K: int, group: int) -> int:
 
 
 def bpdq_pack(bits: np.ndarray, coef: np.ndarray, group: int) -> np.ndarray:
-    """bits uint8 [K][out][in], coef uint16 [K+1][out][in/group] -> blob (uint8 array)."""
+    """bits uint8 [K][out][in], coef uint16 [K+1][out][ceil(in/group)] -> blob (uint8 array)."""
     bits = np.ascontiguousarray(bits, dtype=np.uint8)
     coef = np.ascontiguousarray(coef, dtype=np.uint16)
     K, out, in_ = bits.shape
-    if coef.shape != (K + 1, out, in_ // group):
+    if coef.shape != (K + 1, out, -(-in_ // group)):
         raise ValueError(f"coef shape {coef.shape} does not match bits {bits.shape} with group {group}")
     n = bpdq_packed_bytes(out, in_, K, group)
     if n == 0:
@@ -113,17 +113,17 @@ def bpdq_unpack(blob: np.ndarray, out: int, in_: int, K: int, group: int):
     if blob.size != bpdq_packed_bytes(out, in_, K, group) or blob.size == 0:
         raise BpdqError(ERR_INVALID, "blob size does not match the shape")
     bits = np.empty((K, out, in_), dtype=np.uint8)
-    coef = np.empty((K + 1, out, in_ // group), dtype=np.uint16)
+    coef = np.empty((K + 1, out, -(-in_ // group)), dtype=np.uint16)
     _check(lib().bpdq_unpack(_np_ptr(blob), out, in_, K, group, _np_ptr(bits), _np_ptr(coef)))
     return bits, coef
 
 
 def bpdq_quantize_datafree(w: np.ndarray, K: int, group: int, alpha: float = 1e-4):
-    """w float32 [out][in] -> (bits uint8 [K][out][in], coef uint16 [K+1][out][in/group])."""
+    """w float32 [out][in] -> (bits uint8 [K][out][in], coef uint16 [K+1][out][ceil(in/group)])."""
     w = np.ascontiguousarray(w, dtype=np.float32)
     out, in_ = w.shape
     bits = np.empty((K, out, in_), dtype=np.uint8)
-    coef = np.empty((K + 1, out, in_ // group), dtype=np.uint16)
+    coef = np.empty((K + 1, out, -(-in_ // group)), dtype=np.uint16)
     _check(lib().bpdq_quantize_datafree(_np_ptr(w), out, in_, K, group, alpha, _np_ptr(bits), _np_ptr(coef)))
     return bits, coef
 
@@ -134,7 +134,7 @@ def bpdq_truncate_planes(bits: np.ndarray, coef: np.ndarray, group: int, K2: int
     coef = np.ascontiguousarray(coef, dtype=np.uint16)
     K, out, in_ = bits.shape
     bits2 = np.empty((K2, out, in_), dtype=np.uint8)
-    coef2 = np.empty((K2 + 1, out, in_ // group), dtype=np.uint16)
+    coef2 = np.empty((K2 + 1, out, -(-in_ // group)), dtype=np.uint16)
     _check(lib().bpdq_truncate_planes(_np_ptr(bits), _np_ptr(coef), out, in_, K, group, K2, _np_ptr(bits2), _np_ptr(coef2)))
     return bits2, coef2
 

@@ -66,7 +66,7 @@ __global__ void fill_planes_kernel(uint8_t* __restrict__ blob, unsigned long lon
 
 __global__ void fill_coefs_kernel(uint8_t* __restrict__ cbase, unsigned long long key, int out, int in,
                                   int K, int group) {
-    const long long ngroups = in / group;
+    const long long ngroups = (in + group - 1) / group;
     const long long total = ngroups * (K + 1) * (long long)out;
     // binary32 constants identical to the host generator's
     const float c0_scale = 0x1.47ae14p-6f * 0x1p-16f;

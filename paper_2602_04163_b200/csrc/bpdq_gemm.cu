@@ -658,7 +658,7 @@ int ensure_packed_maps(bpdq_handle_s* h, EncodeTiledFn enc) {
     const cuuint64_t pd[2] = {(cuuint64_t)h->out * 2, (cuuint64_t)(h->in / 128) * K};
     const cuuint64_t ps[1] = {(cuuint64_t)h->out * 16};
     const cuuint32_t pb[2] = {(cuuint32_t)BM * 2, (cuuint32_t)K};
-    const cuuint64_t cd[2] = {(cuuint64_t)h->out / 4, (cuuint64_t)(h->in / h->group) * (K + 1)};
+    const cuuint64_t cd[2] = {(cuuint64_t)h->out / 4, (cuuint64_t)((h->in + h->group - 1) / h->group) * (K + 1)};
     const cuuint64_t cs[1] = {(cuuint64_t)h->out * 2};
     const cuuint32_t cb[2] = {(cuuint32_t)BM / 4, (cuuint32_t)(ng * (K + 1))};
     CUresult r1 = enc(reinterpret_cast<CUtensorMap*>(h->gemm_maps[0]), CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, h->d_blob, pd, ps, pb, estr,

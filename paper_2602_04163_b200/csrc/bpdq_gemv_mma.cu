@@ -572,7 +572,7 @@ int few_prepare(bpdq_handle_s* h) {
     const cuuint64_t pd[3] = {16, (cuuint64_t)(h->in / 128) * K, (cuuint64_t)h->out / 8};
     const cuuint64_t ps[2] = {(cuuint64_t)h->out * 16, 128};
     const cuuint32_t pb[3] = {16, (cuuint32_t)(4 * K), (cuuint32_t)rows / 8};
-    const cuuint64_t cd[2] = {(cuuint64_t)h->out / 4, (cuuint64_t)(h->in / h->group) * (K + 1)};
+    const cuuint64_t cd[2] = {(cuuint64_t)h->out / 4, (cuuint64_t)((h->in + h->group - 1) / h->group) * (K + 1)};
     const cuuint64_t cs[1] = {(cuuint64_t)h->out * 2};
     const cuuint32_t cb[2] = {(cuuint32_t)rows / 4, (cuuint32_t)(ngs * (K + 1))};
     const CUresult r1 = enc(&maps[0], CU_TENSOR_MAP_DATA_TYPE_UINT64, 3, h->d_blob, pd, ps, pb, estr3, CU_TENSOR_MAP_INTERLEAVE_NONE,

@@ -27,7 +27,7 @@ BPDQ_HD size_t coef_offset(int64_t G, int i, int64_t r, int K, int64_t out) {
 }
 BPDQ_HD size_t planes_bytes(int64_t out, int64_t in, int K) { return (size_t)(out * in * K / 8); }
 BPDQ_HD size_t coefs_bytes(int64_t out, int64_t in, int K, int64_t g) {
-    return (size_t)(out * (in / g) * (K + 1) * 2);
+    return (size_t)(out * ((in + g - 1) / g) * (K + 1) * 2);   // ceil(in / g) groups: the last one may be short
 }
 
 bool shape_supported(int out, int in, int K, int group);

@@ -24,7 +24,7 @@ bool shape_supported(int out, int in, int K, int group) {
     if (out <= 0 || in <= 0) return false;
     if (K < 1 || K > 4) return false;
     if (group != 64 && group != 128 && group != 256) return false;
-    if (in % kBlockCols || in % group) return false;
+    if (in % kBlockCols) return false;                // whole 128-column blocks; with g = 256 the last group may hold 128 columns
     if (out % 16) return false;
     return true;
 }
@@ -47,7 +47,7 @@ extern "C" int bpdq_pack(const uint8_t* bits, const uint16_t* coef, int out, int
         return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_pack: unsupported shape out=%d in=%d K=%d g=%d",
                          out, in, K, group);
     uint8_t* dst = static_cast<uint8_t*>(blob);
-    const int64_t nblocks = in / kBlockCols, ngroups = in / group;
+    const int64_t nblocks = in / kBlockCols, ngroups = (in + group - 1) / group;
     for (int i = 0; i < K; ++i) {
         for (int64_t r = 0; r < out; ++r) {
             const uint8_t* row = bits + ((int64_t)i * out + r) * in;
@@ -84,7 +84,7 @@ extern "C" int bpdq_unpack(const void* blob, int out, int in, int K, int group, 
         return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_unpack: unsupported shape out=%d in=%d K=%d g=%d",
                          out, in, K, group);
     const uint8_t* src = static_cast<const uint8_t*>(blob);
-    const int64_t nblocks = in / kBlockCols, ngroups = in / group;
+    const int64_t nblocks = in / kBlockCols, ngroups = (in + group - 1) / group;
     for (int i = 0; i < K; ++i)
         for (int64_t r = 0; r < out; ++r) {
             uint8_t* row = bits + ((int64_t)i * out + r) * in;

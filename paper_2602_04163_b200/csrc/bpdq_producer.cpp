@@ -58,7 +58,7 @@ bool solve_small(double (&N)[5][5], double (&rhs)[5], int n, double (&c)[5]) {
 extern "C" int bpdq_quantize_datafree(const float* w, int out, int in, int K, int group, double alpha, uint8_t* bits,
                                       uint16_t* coef) {
     if (!w || !bits || !coef) return set_error(BPDQ_ERR_INVALID, "bpdq_quantize_datafree: null pointer");
-    if (!shape_supported(out, in, K, group))
+    if (!shape_supported(out, in, K, group) || in % group)          // the fit works on whole groups
         return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_quantize_datafree: unsupported shape out=%d in=%d K=%d g=%d", out, in, K, group);
     if (!(alpha >= 0.0)) return set_error(BPDQ_ERR_INVALID, "bpdq_quantize_datafree: alpha must be >= 0");
     const int64_t ng = in / group;
@@ -110,7 +110,7 @@ extern "C" int bpdq_quantize_datafree(const float* w, int out, int in, int K, in
 extern "C" int bpdq_truncate_planes(const uint8_t* bits, const uint16_t* coef, int out, int in, int K, int group, int K2,
                                     uint8_t* bits2, uint16_t* coef2) {
     if (!bits || !coef || !bits2 || !coef2) return set_error(BPDQ_ERR_INVALID, "bpdq_truncate_planes: null pointer");
-    if (!shape_supported(out, in, K, group) || K2 < 1 || K2 > K)
+    if (!shape_supported(out, in, K, group) || in % group || K2 < 1 || K2 > K)
         return set_error(BPDQ_ERR_UNSUPPORTED, "bpdq_truncate_planes: unsupported shape out=%d in=%d K=%d g=%d K2=%d", out, in, K, group, K2);
     const int drop = K - K2;
     const int64_t plane = (int64_t)out * in, ng = in / group, cplane = (int64_t)out * ng;

@@ -111,11 +111,9 @@ def plane_bits(seed: int, out: int, in_: int, K: int, rows=None) -> np.ndarray:
 
 
 def coefficients(seed: int, out: int, in_: int, K: int, group: int, rows=None) -> np.ndarray:
-    """fp16 bit patterns, uint16 [K+1][len(rows)][in/group]; index 0 is the offset c0."""
-    if in_ % group:
-        raise ValueError("in must be a multiple of group")
+    """fp16 bit patterns, uint16 [K+1][len(rows)][ceil(in/group)]; index 0 is the offset c0 (a last group may be short)."""
     r = _rows(out, rows)
-    ng = in_ // group
+    ng = -(-in_ // group)
     res = np.empty((K + 1, r.size, ng), dtype=np.uint16)
     g = np.arange(ng, dtype=np.uint64)[None, :]
     for i in range(K + 1):

@@ -10,7 +10,8 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("K,g,out,in_", [(2, 128, 160, 640), (3, 128, 96, 384), (1, 128, 32, 128),
-                                          (4, 128, 48, 256), (2, 64, 80, 384), (3, 256, 64, 768), (2, 128, 16, 128)])
+                                          (4, 128, 48, 256), (2, 64, 80, 384), (3, 256, 64, 768), (2, 128, 16, 128),
+                                          (2, 256, 160, 640), (3, 256, 272, 1152)])   # g = 256 with a short last group (2.5 and 4.5 groups)
 def test_dequant_bit_exact(K, g, out, in_):
     h, bits, coef = G.make_layer(10 + K, out, in_, K, g)
     w = G.run_dequant(h)
@@ -31,9 +32,9 @@ def test_dequant_adversarial_coefficients():
     assert np.array_equal(G.run_dequant(h), oracle.dequant(bits, coef, g))
 
 
-@pytest.mark.parametrize("K,g", [(2, 128), (3, 128), (4, 64)])
-def test_device_generator_matches_host_generator(K, g):
-    out, in_ = 96, 512
+@pytest.mark.parametrize("K,g,in_", [(2, 128, 512), (3, 128, 512), (4, 64, 512), (2, 256, 640)])
+def test_device_generator_matches_host_generator(K, g, in_):
+    out = 96
     h = binding.Handle(out, in_, K, g, None, 77, 1)
     blob = h.bpdq_read_blob()
     bits, coef = oracle.unpack(blob, out, in_, K, g)

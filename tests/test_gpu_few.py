@@ -28,6 +28,8 @@ pytestmark = pytest.mark.gpu
     (2, 128, 1040, 8192, 16),     # sixteen slices: four column ranges accumulate through the workspace
     (4, 128, 2064, 2048, 16),     # sixteen candidates with tasks of two row groups: several segments per CTA, ragged last task
     (4, 64, 1040, 4096, 20),      # the same with two token tiles and a coefficient group per half block
+    (2, 256, 160, 640, 7),        # g = 256 with a short last group (the last slice holds one block of it)
+    (3, 256, 272, 1152, 20),      # four and a half groups, two token tiles
 ])
 def test_few_token_kernel(K, g, out, in_, M):
     h, bits, coef = G.make_layer(140 + K, out, in_, K, g, max_M=M)

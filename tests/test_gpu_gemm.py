@@ -27,6 +27,9 @@ pytestmark = pytest.mark.gpu
     (4, 128, 384, 2048, 7),      # two-way split, ragged token tile
     (2, 128, 256, 4096, 100),    # 128-token tile shared by four CTAs (split over the input dimension), two CTAs per SM
     (3, 128, 384, 2048, 128),    # 128-token tile, two-way split, all 128 token columns in use
+    (2, 256, 160, 640, 24),      # g = 256 with a short last group: tile kernel
+    (3, 256, 272, 1152, 200),    # ... 256-token kernel
+    (2, 256, 160, 1664, 600),    # ... 512-token kernel (six and a half groups)
     (2, 128, 256, 384, 20500),   # 162 output tiles for 148 persistent CTAs: a second tile per CTA, odd number of blocks per tile
     (4, 128, 128, 640, 38000),   # 149 tiles, three-stage ring (K = 4), odd number of blocks per tile
     (3, 64, 160, 640, 24),       # tile kernel, ragged last row tile (the tensor maps fill the missing rows), two groups per block

@@ -52,6 +52,8 @@ def test_m_zero_and_bad_arguments():
     (3, 64, 272, 896, 2),        # W3-G64, two tokens
     (4, 64, 48, 1536, 3),
     (1, 64, 1024, 2048, 1),
+    (2, 256, 160, 640, 1),       # g = 256, two and a half groups: the last group is short (and so is the second slice)
+    (3, 256, 272, 1152, 2),      # four and a half groups
 ])
 def test_lut_kernel(K, g, out, in_, M):
     h, bits, coef = G.make_layer(40 + K, out, in_, K, g, max_M=M)

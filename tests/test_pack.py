@@ -37,6 +37,19 @@ def test_one_hot_bits_land_where_the_layout_says():
         assert nz[0] == ((b * K + i) * out + r) * 16 + p and blob[nz[0]] == 1 << t
 
 
+def test_round_trip_with_a_short_last_group():
+    K, g, out, in_ = 2, 256, 32, 640                     # two and a half groups
+    bits = synth.plane_bits(21, out, in_, K)
+    coef = synth.coefficients(21, out, in_, K, g)
+    assert coef.shape == (K + 1, out, 3)
+    blob = binding.bpdq_pack(bits, coef, g)
+    assert blob.size == binding.bpdq_packed_bytes(out, in_, K, g) == out * in_ * K // 8 + out * 3 * (K + 1) * 2
+    b2, c2 = binding.bpdq_unpack(blob, out, in_, K, g)
+    assert np.array_equal(b2, bits) and np.array_equal(c2, coef)
+    b3, c3 = oracle.unpack(blob, out, in_, K, g)          # the checker's own reader agrees
+    assert np.array_equal(b3, bits) and np.array_equal(c3, coef)
+
+
 def test_coefficient_placement():
     K, g, out, in_ = 3, 64, 16, 128
     bits = np.zeros((K, out, in_), dtype=np.uint8)
@@ -93,7 +106,7 @@ def test_rejects_bad_input():
     assert binding.bpdq_packed_bytes(128, 200, 2, 128) == 0       # in % 128
     assert binding.bpdq_packed_bytes(128, 256, 5, 128) == 0
     assert binding.bpdq_packed_bytes(128, 256, 2, 32) == 0
-    assert binding.bpdq_packed_bytes(128, 384, 2, 256) == 0       # in % g
+    assert binding.bpdq_packed_bytes(128, 384, 2, 256) == 128 * 384 * 2 // 8 + 128 * 2 * 3 * 2      # one and a half groups: the last one is short
     bits = np.zeros((2, 16, 128), dtype=np.uint8)
     bits[1, 3, 5] = 2
     with pytest.raises(binding.BpdqError) as ei:
