@@ -390,6 +390,8 @@ def run_cuda(args, rank: int, world: int, local_rank: int):
         line["sections"] = extra_sections(torch, binding, args, peaks, sp, stream)
         line["sections"]["seven_separate_calls"] = separate
         line["sections"]["decode_sweep_80_layers_K2"] = full_stack_section(torch, binding, peaks, sp, stream)
+        # the paper's headline deployment format (W2-G256 on the 72B model) as a whole stack
+        line["sections"]["decode_sweep_80_layers_W2-G256"] = full_stack_section(torch, binding, peaks, sp, stream, group=256)
         dg = line["sections"].get("gemv_layer_batched_decoder_groups_K2", {})
         line["config"]["same_layer_other_issue_orders"] = {
             "decoder_legal_groups_qkv_o_gateup_down": {"us_per_layer": dg.get("us_per_layer"), "frac_measured": dg.get("frac_measured")},
@@ -771,13 +773,14 @@ def extra_sections(torch, binding, args, peaks, sp, stream):
     return out
 
 
-def full_stack_section(torch, binding, peaks, sp, stream, n_layers=80):
-    """All linears of an 80-layer 72B-shaped stack (K = 2, about 20.8 GB packed), one token through each."""
+def full_stack_section(torch, binding, peaks, sp, stream, n_layers=80, group=GROUP):
+    """All linears of an 80-layer 72B-shaped stack (K = 2: about 20.8 GB packed at g = 128, 19.2 GB at g = 256), one token
+    through each."""
     shapes, K = synth.QWEN25_72B_LAYER, 2
     hs = []
     for layer in range(n_layers):
         for li, (_, o, i) in enumerate(shapes):
-            hs.append(binding.Handle(o, i, K, GROUP, None, synth.linear_seed(5, layer, li, K), 1))
+            hs.append(binding.Handle(o, i, K, group, None, synth.linear_seed(5, layer, li, K), 1))
     xs = {i: torch.from_numpy(synth.activations(9, 1, i).view(np.int16).copy()).cuda().view(torch.float16) for i in (8192, 29568)}
     ys = {o: torch.empty((1, o), dtype=torch.float16, device="cuda") for o in sorted({o for _, o, _ in shapes})}
 
@@ -786,8 +789,8 @@ def full_stack_section(torch, binding, peaks, sp, stream, n_layers=80):
             h.bpdq_linear(xs[h.in_].data_ptr(), ys[h.out].data_ptr(), 1, sp)
     sweep()
     ms = sorted(event_time_ms(torch, sweep, stream) for _ in range(3))[1]
-    b = n_layers * layer_bytes(shapes, K, 1)
-    res = {"layers": n_layers, "linears": len(hs), "packed_gb": sum(h.packed_bytes for h in hs) / 1e9, "ms_per_sweep": ms,
+    b = n_layers * sum(useful_bytes(o, i, K, group, 1) for _, o, i in shapes)
+    res = {"layers": n_layers, "group": group, "linears": len(hs), "packed_gb": sum(h.packed_bytes for h in hs) / 1e9, "ms_per_sweep": ms,
            "gbs": b / (ms * 1e-3) / 1e9, "frac_measured": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
 
     # the same sweep as one bpdq_linear_batch call per layer (every linear of a batch needs an output of its own)
@@ -803,6 +806,17 @@ def full_stack_section(torch, binding, peaks, sp, stream, n_layers=80):
     ms_b = sorted(event_time_ms(torch, sweep_batched, stream) for _ in range(3))[1]
     res["one_launch_per_layer"] = {"launches": n_layers, "ms_per_sweep": ms_b, "gbs": b / (ms_b * 1e-3) / 1e9,
                                    "frac_measured": b / (ms_b * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    # and in the grouping a decoder allows: {q, k, v} {o} {gate, up} {down}, four launches per layer
+    groups = [[0, 1, 2], [3], [4, 5], [6]]
+
+    def sweep_groups():
+        for layer in range(n_layers):
+            for grp in groups:
+                binding.bpdq_linear_batch([hs[layer * n + j] for j in grp], [x_ptrs[j] for j in grp], [y_ptrs[j] for j in grp], 1, sp)
+    sweep_groups()
+    ms_g = sorted(event_time_ms(torch, sweep_groups, stream) for _ in range(3))[1]
+    res["decoder_groups"] = {"launches": n_layers * len(groups), "ms_per_sweep": ms_g, "gbs": b / (ms_g * 1e-3) / 1e9,
+                             "frac_measured": b / (ms_g * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     for h in hs:
         h.bpdq_destroy()
     return res
