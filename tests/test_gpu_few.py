@@ -96,3 +96,19 @@ def test_few_token_kernel_rejects_what_it_cannot_take():
     with pytest.raises(binding.BpdqError) as ei:
         h.bpdq_linear_ex(x.data_ptr(), y.data_ptr(), binding.FEW_MAX_M + 1, binding.KERNEL_FEW, G.stream_ptr())
     assert ei.value.code == binding.ERR_INVALID and h.bpdq_launch_count() == n0
+
+
+@pytest.mark.parametrize("g", [128, 64])
+def test_dispatcher_with_sixteen_candidates(g):
+    """K = 4 through bpdq_linear at the token counts either side of its thresholds (look-up-table kernel up to 3 tokens,
+    2 at g = 64; few-token kernel to 16; tcgen05 beyond): every choice within the checker's bound."""
+    K, out, in_ = 4, 272, 1536
+    h, bits, coef = G.make_layer(190 + g, out, in_, K, g, max_M=20)
+    for M in (1, 2, 3, 4, 16, 17):
+        x = synth.activations(191 + M, M, in_)
+        n0 = h.bpdq_launch_count()
+        G.check_linear(h, bits, coef, x, g, binding.KERNEL_AUTO, what=f"K=4 g={g} M={M}")
+        lut_max = 2 if g == 64 else 3
+        passes = (M + 1) // 2 if M <= lut_max else 1      # the look-up-table kernel takes two tokens per pass
+        assert h.bpdq_launch_count() - n0 == passes
+    h.bpdq_destroy()
